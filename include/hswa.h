@@ -1,0 +1,162 @@
+/*
+ * hswa.h -- C ABI of the hybrid sliding-window / full attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the attention hot path of a layer stack that interleaves Sliding Window Attention
+ * layers (window W, 128 in the paper) with Full Attention layers (paper Sec. 2.1), over the dual-pool KV
+ * cache of paper Sec. 3.1.1: Full layers keep the whole sequence in pages reached through a per-request
+ * block table (equal prefixes may share physical pages, Sec. 3.1.3); SWA layers keep strictly O(W) KV per
+ * request in a ring of R pages reached through a ring table and a ring head.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device addresses on the current device; "host" pointers are ordinary
+ *     host memory.  Every array is caller-owned; the library never frees or keeps caller memory.
+ *   - Every call that takes `stream` (a cudaStream_t passed as void*) is asynchronous on that stream and
+ *     returns after the launches are queued.  No call synchronises except hswa_get_async_error,
+ *     hswa_create and hswa_destroy.
+ *   - The library allocates exactly one 16-byte device error word per handle (hswa_create) and nothing
+ *     else; scratch memory is a caller-provided workspace (hswa_workspace_bytes).
+ *   - Host-detectable misuse returns a status at once and launches nothing.  Device-detectable misuse
+ *     (hswa_validate_batch; bounded waits inside kernels) is recorded in the error word, the offending
+ *     access is skipped, and the kernel returns normally: nothing traps, asserts or spins without bound.
+ *   - No global mutable state; a handle may be used from one thread at a time.
+ *
+ * Symbols (bf16 everywhere KV or Q are stored):
+ *   Hq, Hkv query / KV heads, G = Hq / Hkv (query head h uses KV head h / G), D head_dim, P page_size,
+ *   W window, R ring_pages, C = R * P ring slots, B batch, ctx[r] tokens cached before the step,
+ *   n[r] new tokens of request r in the step, T = sum n[r], p = ctx[r] + i the absolute position of the
+ *   i-th new token.
+ *
+ * Pool layout (one pool per layer): bf16 [num_pages][2][Hkv][P][D], index 1 being 0 = K, 1 = V, so a
+ * (page, K|V, head) slab is P * D contiguous elements.  The pool base must be 256-byte aligned (TMA
+ * descriptors are built over it); q, k_new, v_new and out must be 16-byte aligned.
+ *
+ * Position -> storage (Sec. 3.1.1, "Full index authoritative, Full -> SWA mapping"):
+ *   Full layer: page = block_table[r][p / P], slot = p % P.
+ *   SWA  layer: s = (ring_head[r] + (p - ctx[r])) mod C (mathematical mod),
+ *               page = ring_table[r][s / P], slot = s % P.
+ * Attention (plain softmax attention over the logical sequence; the cache is only storage):
+ *   keys j in [lo, p], lo = 0 on a Full layer and max(0, p - W + 1) on an SWA layer (W keys including the
+ *   query's own position); out = softmax(sm_scale * q K^T) V with fp32 accumulation, lse = natural-log
+ *   log-sum-exp of the scaled scores.
+ *
+ * Supported shapes: D in {64, 128}; P in {16, 32, 64}; 1 <= G <= 8; W >= 1; R * P >= W + 1.
+ */
+#ifndef HSWA_H_
+#define HSWA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hswa_handle hswa_handle; /* opaque */
+
+typedef enum {
+  HSWA_OK = 0,
+  HSWA_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent fields */
+  HSWA_ERR_UNSUPPORTED = 2, /* shape outside the supported set */
+  HSWA_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  HSWA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed, or no sm_100 device */
+  HSWA_ERR_BOUNDS = 5,      /* device-side validation found an out-of-range id or length */
+  HSWA_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel ran out */
+} hswa_status;
+
+/* Immutable per model. */
+typedef struct {
+  int32_t num_q_heads;  /* Hq */
+  int32_t num_kv_heads; /* Hkv, divides Hq */
+  int32_t head_dim;     /* D */
+  int32_t page_size;    /* P */
+  int32_t window;       /* W (paper: 128) */
+  int32_t ring_pages;   /* R; 0 selects ceil(W / P) + 1 */
+  float sm_scale;       /* 0 selects 1 / sqrt(D) */
+  int32_t out_dtype;    /* 0 = bf16 output, 1 = fp32 output */
+} hswa_config;
+
+/* One layer's cache.  `pool` is a device pointer, caller-owned, layout above. */
+typedef struct {
+  void* pool;
+  int64_t num_pages;
+  int32_t is_swa; /* per-layer flag: 1 = SWA layer (ring storage, window mask), 0 = Full layer */
+} hswa_layer;
+
+/* One step's batch.  All arrays are DEVICE pointers, caller-owned, constant during the step (every layer
+ * of the step reuses them); only hswa_step_advance changes ctx_len / ring_head. */
+typedef struct {
+  int32_t batch;              /* B >= 0 */
+  const int32_t* ctx_len;     /* [B] tokens cached before this step */
+  const int32_t* q_indptr;    /* [B+1] prefix sums of n[r]; NULL means n[r] = 1 for all r (decode) */
+  const int32_t* block_table; /* [B][max_blocks] page ids valid in every Full layer's pool */
+  int32_t max_blocks;
+  const int32_t* ring_table; /* [B][R] page ids valid in every SWA layer's pool */
+  const int32_t* ring_head;  /* [B] ring slot in [0, C) of position ctx_len[r] (the next write) */
+  int32_t max_q_len;         /* host-known upper bound of n[r]   (launch geometry only) */
+  int32_t total_q;           /* T, host-known                      */
+  int32_t max_ctx_len;       /* host-known upper bound of ctx_len[r] (launch geometry only) */
+} hswa_batch;
+
+/* Create / destroy a handle on the current CUDA device.  hswa_create validates the config (status
+ * UNSUPPORTED / INVALID_ARG), checks the device is compute capability 10.x and allocates the error word.
+ * Both calls synchronise the device.  `cfg` is a host pointer and is copied. */
+hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out);
+void hswa_destroy(hswa_handle* h);
+
+/* Bytes of workspace (device memory, 256-byte aligned, caller-owned) that hswa_decode_attn and
+ * hswa_prefill_attn need for batches bounded by the three arguments.  Pure host arithmetic. */
+size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max_total_q, int32_t max_ctx_len);
+
+/* Debug aid: checks on the device, for the given layer kind, that every id and length the step would use
+ * is in range (0 <= ctx, n >= 0, block-table coverage of ctx + n, page ids < num_pages, ring_head in
+ * [0, C)).  The first violation is recorded in the error word as {HSWA_ERR_BOUNDS, request, index, value}. */
+hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, void* stream);
+
+/* KV append (Sec. 3.1.1 pools; Sec. 3.1.3: an SWA pool stays at window magnitude).
+ * k_new, v_new: device, bf16 [T][Hkv][D].  Token i of request r is written at the storage location of
+ * position ctx[r] + i.  On an SWA layer later tokens overwrite earlier ones, so only the last min(n, C)
+ * tokens of a request are written.  Nothing else in the pool changes.
+ * Caller guarantees that pages receiving an append are not shared with another request. */
+hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* k_new,
+                           const void* v_new, void* stream);
+
+/* Batched GQA decode attention, one new token per request (batch->q_indptr must be NULL).
+ * q: device bf16 [B][Hq][D].  out: device [B][Hq][D] in cfg.out_dtype.  lse: device fp32 [B][Hq] or NULL.
+ * k_new, v_new: device bf16 [B][Hkv][D], or both NULL.
+ *   non-NULL: the new token's K/V are appended (fused into the attention kernel) and attended to.
+ *   NULL:     the caller already ran hswa_kv_append with the same un-advanced batch; position ctx[r] is
+ *             read from the cache.
+ * Full layers split the key range over thread blocks (split-K) and merge the partial results; partials
+ * live in `workspace`. */
+hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* q,
+                             const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
+/* Chunked prefill attention: request r extends its cached context by n[r] new tokens.
+ * q: device bf16 [T][Hq][D]; k_new, v_new: device bf16 [T][Hkv][D] (required); out: device [T][Hq][D];
+ * lse: device fp32 [T][Hq] or NULL.
+ * Keys j < ctx[r] are read from the cache AS IT IS BEFORE THIS CHUNK'S APPEND (pages on a Full layer; the
+ * ring on an SWA layer), keys j >= ctx[r] from k_new / v_new.  Causal mask on Full layers, causal + window
+ * mask on SWA layers; key tiles wholly outside the mask are skipped.
+ * fuse_append != 0: the chunk's K/V are also appended to the cache, ordered after every read of the old
+ * ring contents (an SWA chunk longer than C - W + 1 tokens overwrites ring slots its own first queries
+ * need, so "append, then attend" is not available on SWA layers). */
+hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* q,
+                              const void* k_new, const void* v_new, int32_t fuse_append, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step advance, once per step after all layers: ctx_len[r] += n[r], ring_head[r] = (ring_head[r] + n[r])
+ * mod C.  ctx_len, ring_head: device int32 [B], updated in place.  q_indptr: device or NULL (n = 1). */
+hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
+                              const int32_t* q_indptr, void* stream);
+
+/* Synchronises `stream`, copies the error word to info[4] = {status, request, index, value} (host), clears
+ * it, and returns info[0] as a status (HSWA_OK when nothing was recorded). */
+hswa_status hswa_get_async_error(hswa_handle* h, void* stream, int32_t info[4]);
+
+const char* hswa_status_string(hswa_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HSWA_H_ */

@@ -1,0 +1,318 @@
+// Host side of the C ABI: argument validation, launch planning, TMA descriptor construction, dispatch.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "hswa_internal.cuh"
+
+namespace {
+
+constexpr int kMinSplitLen = 256;
+constexpr int kMaxSplitLen = 2048;
+
+ModelParams model_params(const hswa_handle* h) {
+  ModelParams m;
+  m.Hq = h->cfg.num_q_heads;
+  m.Hkv = h->cfg.num_kv_heads;
+  m.G = h->group;
+  m.D = h->cfg.head_dim;
+  m.P = h->cfg.page_size;
+  m.W = h->cfg.window;
+  m.R = h->cfg.ring_pages;
+  m.C = h->ring_slots;
+  m.scale_log2 = h->cfg.sm_scale * 1.4426950408889634f;
+  m.out_fp32 = h->cfg.out_dtype;
+  return m;
+}
+
+BatchParams batch_params(const hswa_batch* b) {
+  BatchParams o;
+  o.B = b->batch;
+  o.ctx_len = b->ctx_len;
+  o.q_indptr = b->q_indptr;
+  o.block_table = b->block_table;
+  o.max_blocks = b->max_blocks;
+  o.ring_table = b->ring_table;
+  o.ring_head = b->ring_head;
+  return o;
+}
+
+// Checks every host-visible field of a (layer, batch) pair.
+hswa_status check_common(const hswa_handle* h, const hswa_layer* layer, const hswa_batch* b) {
+  if (!h || !layer || !b) return HSWA_ERR_INVALID_ARG;
+  if (b->batch < 0 || b->total_q < 0 || b->max_q_len < 0 || b->max_ctx_len < 0) return HSWA_ERR_INVALID_ARG;
+  if (b->batch == 0) return HSWA_OK;
+  if (!layer->pool || layer->num_pages <= 0) return HSWA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(layer->pool) & 255) != 0) return HSWA_ERR_INVALID_ARG;
+  if (layer->num_pages > (int64_t)INT32_MAX) return HSWA_ERR_UNSUPPORTED;
+  if (!b->ctx_len) return HSWA_ERR_INVALID_ARG;
+  if (layer->is_swa) {
+    if (!b->ring_table || !b->ring_head) return HSWA_ERR_INVALID_ARG;
+  } else {
+    if (!b->block_table || b->max_blocks <= 0) return HSWA_ERR_INVALID_ARG;
+  }
+  if (b->q_indptr == nullptr && (b->total_q != b->batch || b->max_q_len != 1)) return HSWA_ERR_INVALID_ARG;
+  if (b->max_q_len > b->total_q) return HSWA_ERR_INVALID_ARG;
+  return HSWA_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// Keys per split for Full-layer decode: long enough that the partial (m, l, o) traffic stays below one
+// percent of the KV bytes, short enough that the grid fills the machine.
+int plan_split_len(const hswa_handle* h, int batch, int max_ctx_len) {
+  const long long kv_len = (long long)max_ctx_len + 1;
+  int len = kMaxSplitLen;
+  const long long want = 4LL * h->num_sms;
+  while (len > kMinSplitLen && (long long)batch * h->cfg.num_kv_heads * ((kv_len + len - 1) / len) < want) len >>= 1;
+  return len;
+}
+
+int plan_max_splits(int split_len, int max_ctx_len) {
+  const long long kv_len = (long long)max_ctx_len + 1;
+  return (int)((kv_len + split_len - 1) / split_len);
+}
+
+// 4-D view of a pool for TMA: {D, P, 2 * Hkv, num_pages}, box {64, P, 1, 1}, 128-byte swizzle.
+hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtensorMap* tm) {
+  const hswa_config& c = h->cfg;
+  cuuint64_t dims[4] = {(cuuint64_t)c.head_dim, (cuuint64_t)c.page_size, (cuuint64_t)(2 * c.num_kv_heads),
+                        (cuuint64_t)layer->num_pages};
+  cuuint64_t strides[3] = {(cuuint64_t)c.head_dim * 2, (cuuint64_t)c.head_dim * 2 * c.page_size,
+                           (cuuint64_t)c.head_dim * 2 * c.page_size * 2 * c.num_kv_heads};
+  cuuint32_t box[4] = {64, (cuuint32_t)c.page_size, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult rc = h->encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, layer->pool, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hswa_status_string(hswa_status s) {
+  switch (s) {
+    case HSWA_OK: return "ok";
+    case HSWA_ERR_INVALID_ARG: return "invalid argument";
+    case HSWA_ERR_UNSUPPORTED: return "unsupported shape";
+    case HSWA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case HSWA_ERR_CUDA: return "CUDA call failed";
+    case HSWA_ERR_BOUNDS: return "device-side bounds violation";
+    case HSWA_ERR_TIMEOUT: return "bounded wait inside a kernel ran out";
+  }
+  return "unknown status";
+}
+
+hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out) {
+  if (!cfg || !out) return HSWA_ERR_INVALID_ARG;
+  *out = nullptr;
+  hswa_config c = *cfg;
+  if (c.num_q_heads <= 0 || c.num_kv_heads <= 0 || c.num_q_heads % c.num_kv_heads != 0) return HSWA_ERR_INVALID_ARG;
+  if (c.window <= 0 || c.page_size <= 0 || c.ring_pages < 0) return HSWA_ERR_INVALID_ARG;
+  if (c.out_dtype != 0 && c.out_dtype != 1) return HSWA_ERR_INVALID_ARG;
+  if (!(c.sm_scale >= 0.f) || std::isinf(c.sm_scale)) return HSWA_ERR_INVALID_ARG;
+  if (c.head_dim != 64 && c.head_dim != 128) return HSWA_ERR_UNSUPPORTED;
+  if (c.page_size != 16 && c.page_size != 32 && c.page_size != 64) return HSWA_ERR_UNSUPPORTED;
+  const int group = c.num_q_heads / c.num_kv_heads;
+  if (group > 8) return HSWA_ERR_UNSUPPORTED;
+  if (c.ring_pages == 0) c.ring_pages = (c.window + c.page_size - 1) / c.page_size + 1;
+  if ((int64_t)c.ring_pages * c.page_size < (int64_t)c.window + 1) return HSWA_ERR_INVALID_ARG;
+  if ((int64_t)c.ring_pages * c.page_size > (1 << 20)) return HSWA_ERR_UNSUPPORTED;
+  if (c.sm_scale == 0.f) c.sm_scale = 1.0f / std::sqrt((float)c.head_dim);
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return HSWA_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (prop.major != 10) return HSWA_ERR_CUDA;  // kernels are built for sm_100a only
+
+  hswa_handle* h = new (std::nothrow) hswa_handle();
+  if (!h) return HSWA_ERR_INVALID_ARG;
+  h->cfg = c;
+  h->ring_slots = c.ring_pages * c.page_size;
+  h->group = group;
+  h->device = dev;
+  h->num_sms = prop.multiProcessorCount;
+  h->err = nullptr;
+  h->encode_tiled = nullptr;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete h;
+    return HSWA_ERR_CUDA;
+  }
+  h->encode_tiled = reinterpret_cast<hswa_encode_tiled_fn>(fn);
+  if (cudaMalloc(&h->err, 4 * sizeof(int32_t)) != cudaSuccess || cudaMemset(h->err, 0, 4 * sizeof(int32_t)) != cudaSuccess ||
+      cudaDeviceSynchronize() != cudaSuccess) {
+    if (h->err) cudaFree(h->err);
+    delete h;
+    return HSWA_ERR_CUDA;
+  }
+  *out = h;
+  return HSWA_OK;
+}
+
+void hswa_destroy(hswa_handle* h) {
+  if (!h) return;
+  cudaDeviceSynchronize();
+  if (h->err) cudaFree(h->err);
+  delete h;
+}
+
+size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max_total_q, int32_t max_ctx_len) {
+  if (!h || max_batch <= 0 || max_ctx_len < 0) return 0;
+  (void)max_total_q;  // prefill needs no scratch
+  // Upper bound of rows * splits over every batch <= max_batch and context <= max_ctx_len under
+  // plan_split_len: at the longest split length a row has ceil(kv / 2048) splits; a shorter length is only
+  // chosen while batch * Hkv * splits stays below twice the fill target.
+  const size_t kv = (size_t)max_ctx_len + 1;
+  const size_t long_splits = (kv + kMaxSplitLen - 1) / kMaxSplitLen + 2;
+  const size_t want = 4 * (size_t)h->num_sms;
+  const size_t row_splits = (size_t)h->cfg.num_q_heads * max_batch * long_splits + 2 * want * h->group;
+  const size_t o_bytes = row_splits * h->cfg.head_dim * sizeof(float);
+  const size_t ml_bytes = row_splits * sizeof(float2);
+  return ((o_bytes + 255) & ~size_t(255)) + ((ml_bytes + 255) & ~size_t(255));
+}
+
+hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, void* stream) {
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  if (cudaSetDevice(h->device) != cudaSuccess) return HSWA_ERR_CUDA;
+  cudaError_t e = hswa_launch_validate(model_params(h), batch_params(b), layer->is_swa, layer->num_pages, h->err,
+                                       (cudaStream_t)stream);
+  return e == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
+hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* k_new,
+                           const void* v_new, void* stream) {
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  if (b->batch == 0 || b->total_q == 0) return HSWA_OK;
+  if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return HSWA_ERR_INVALID_ARG;
+  AppendParams p;
+  p.m = model_params(h);
+  p.b = batch_params(b);
+  p.pool = static_cast<__nv_bfloat16*>(layer->pool);
+  p.num_pages = layer->num_pages;
+  p.is_swa = layer->is_swa;
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.total_q = b->total_q;
+  return hswa_launch_append(p, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
+hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,
+                             const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  if (b->q_indptr != nullptr) return HSWA_ERR_INVALID_ARG;
+  if (b->batch == 0) return HSWA_OK;
+  if (!q || !out || !aligned16(q) || !aligned16(out)) return HSWA_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return HSWA_ERR_INVALID_ARG;
+  if (k_new && (!aligned16(k_new) || !aligned16(v_new))) return HSWA_ERR_INVALID_ARG;
+
+  DecodeParams p;
+  p.m = model_params(h);
+  p.b = batch_params(b);
+  p.pool = static_cast<__nv_bfloat16*>(layer->pool);
+  p.num_pages = layer->num_pages;
+  p.is_swa = layer->is_swa;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.out = out;
+  p.lse = lse;
+  p.err = h->err;
+  p.part_o = nullptr;
+  p.part_ml = nullptr;
+  if (layer->is_swa) {
+    p.split_len = ((h->ring_slots + 63) / 64) * 64;
+    p.max_splits = 1;
+  } else {
+    p.split_len = plan_split_len(h, b->batch, b->max_ctx_len);
+    p.max_splits = plan_max_splits(p.split_len, b->max_ctx_len);
+    if (p.max_splits > 65535) return HSWA_ERR_UNSUPPORTED;
+    if (p.max_splits > 1) {
+      const size_t rows = (size_t)b->batch * h->cfg.num_q_heads;
+      const size_t o_bytes = (rows * p.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
+      const size_t ml_bytes = (rows * p.max_splits * sizeof(float2) + 255) & ~size_t(255);
+      if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < o_bytes + ml_bytes)
+        return HSWA_ERR_WORKSPACE;
+      p.part_o = static_cast<float*>(workspace);
+      p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + o_bytes);
+    }
+  }
+  CUtensorMap tm;
+  st = make_pool_map(h, layer, &tm);
+  if (st != HSWA_OK) return st;
+  if (hswa_launch_decode(h, tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  return HSWA_OK;
+}
+
+hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,
+                              const void* k_new, const void* v_new, int32_t fuse_append, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes, void* stream) {
+  (void)workspace;
+  (void)workspace_bytes;
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  if (b->batch == 0 || b->total_q == 0) return HSWA_OK;
+  if (!q || !out || !k_new || !v_new) return HSWA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return HSWA_ERR_INVALID_ARG;
+  PrefillParams p;
+  p.m = model_params(h);
+  p.b = batch_params(b);
+  p.pool = static_cast<__nv_bfloat16*>(layer->pool);
+  p.num_pages = layer->num_pages;
+  p.is_swa = layer->is_swa;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.out = out;
+  p.lse = lse;
+  p.total_q = b->total_q;
+  p.max_q_len = b->max_q_len;
+  p.err = h->err;
+  if (hswa_launch_prefill_mma(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (fuse_append) {
+    // stream order puts the append after every read of the pre-append ring contents
+    AppendParams a;
+    a.m = p.m;
+    a.b = p.b;
+    a.pool = p.pool;
+    a.num_pages = p.num_pages;
+    a.is_swa = p.is_swa;
+    a.k_new = p.k_new;
+    a.v_new = p.v_new;
+    a.total_q = p.total_q;
+    if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  }
+  return HSWA_OK;
+}
+
+hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
+                              const int32_t* q_indptr, void* stream) {
+  if (!h || batch < 0) return HSWA_ERR_INVALID_ARG;
+  if (batch == 0) return HSWA_OK;
+  if (!ctx_len || !ring_head) return HSWA_ERR_INVALID_ARG;
+  return hswa_launch_advance(model_params(h), batch, ctx_len, ring_head, q_indptr, (cudaStream_t)stream) == cudaSuccess
+             ? HSWA_OK
+             : HSWA_ERR_CUDA;
+}
+
+hswa_status hswa_get_async_error(hswa_handle* h, void* stream, int32_t info[4]) {
+  if (!h || !info) return HSWA_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(info, h->err, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (cudaMemsetAsync(h->err, 0, 4 * sizeof(int32_t), s) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return HSWA_ERR_CUDA;
+  return (hswa_status)info[0];
+}
+
+}  // extern "C"

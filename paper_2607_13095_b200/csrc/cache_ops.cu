@@ -1,0 +1,121 @@
+// Cache bookkeeping kernels: KV append into pages / ring slots (paper Sec. 3.1.1 dual pools; Sec. 3.1.3: an
+// SWA pool stays at window magnitude), step advance of (ctx_len, ring_head), and the debug validator.
+#include "hswa_internal.cuh"
+
+namespace {
+using namespace hswa_dev;
+
+// Request owning new-token row t: largest r with q_indptr[r] <= t (q_indptr null: r = t).
+__device__ __forceinline__ int find_request(const BatchParams& b, int t) {
+  if (b.q_indptr == nullptr) return t;
+  int lo = 0, hi = b.B;  // invariant: q_indptr[lo] <= t < q_indptr[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (b.q_indptr[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// One thread moves one 16-byte chunk of one (token, K|V, head) row.
+__global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
+  const ModelParams& M = p.m;
+  const int chunks_per_row = M.D / 8;
+  const int chunks_per_tok = 2 * M.Hkv * chunks_per_row;
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t total = (int64_t)p.total_q * chunks_per_tok;
+  if (gid >= total) return;
+  const int t = (int)(gid / chunks_per_tok);
+  int c = (int)(gid % chunks_per_tok);
+  const int kv = c / (M.Hkv * chunks_per_row);
+  c -= kv * M.Hkv * chunks_per_row;
+  const int kh = c / chunks_per_row;
+  const int ch = c % chunks_per_row;
+
+  const int r = find_request(p.b, t);
+  const int t0 = p.b.q_indptr ? p.b.q_indptr[r] : r;
+  const int n = p.b.q_indptr ? p.b.q_indptr[r + 1] - t0 : 1;
+  const int i = t - t0;
+  const int ctx = p.b.ctx_len[r];
+  int page, slot;
+  if (!p.is_swa) {
+    const int pos = ctx + i;
+    const int blk = pos / M.P;
+    if (blk >= p.b.max_blocks) return;
+    page = p.b.block_table[(int64_t)r * p.b.max_blocks + blk];
+    slot = pos % M.P;
+  } else {
+    if (n - i > M.C) return;  // overwritten later in this same step: only the last C tokens survive
+    const int s = math_mod(p.b.ring_head[r] + i, M.C);
+    page = p.b.ring_table[(int64_t)r * M.R + s / M.P];
+    slot = s % M.P;
+  }
+  if (page < 0 || page >= p.num_pages) return;
+  const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)t * M.Hkv + kh) * M.D + ch * 8;
+  __nv_bfloat16* dst = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + slot) * M.D + ch * 8;
+  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+}
+
+__global__ void advance_kernel(ModelParams M, int B, int32_t* ctx_len, int32_t* ring_head, const int32_t* q_indptr) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= B) return;
+  const int n = q_indptr ? q_indptr[r + 1] - q_indptr[r] : 1;
+  ctx_len[r] += n;
+  ring_head[r] = math_mod(ring_head[r] + (n % M.C), M.C);
+}
+
+// One block per request; threads scan the table entries the step would touch.
+__global__ void __launch_bounds__(128) validate_kernel(ModelParams M, BatchParams b, int is_swa, int64_t num_pages,
+                                                       int32_t* err) {
+  const int r = blockIdx.x;
+  const int ctx = b.ctx_len[r];
+  const int n = b.q_indptr ? b.q_indptr[r + 1] - b.q_indptr[r] : 1;
+  if (threadIdx.x == 0) {
+    if (ctx < 0) record_error(err, HSWA_ERR_BOUNDS, r, -1, ctx);
+    if (n < 0) record_error(err, HSWA_ERR_BOUNDS, r, -2, n);
+  }
+  if (ctx < 0 || n < 0) return;
+  if (!is_swa) {
+    const int64_t need = ((int64_t)ctx + n + M.P - 1) / M.P;
+    if (need > b.max_blocks) {
+      if (threadIdx.x == 0) record_error(err, HSWA_ERR_BOUNDS, r, -3, (int)need);
+      return;
+    }
+    for (int i = threadIdx.x; i < need; i += blockDim.x) {
+      const int pg = b.block_table[(int64_t)r * b.max_blocks + i];
+      if (pg < 0 || pg >= num_pages) record_error(err, HSWA_ERR_BOUNDS, r, i, pg);
+    }
+  } else {
+    if (threadIdx.x == 0) {
+      const int hd = b.ring_head[r];
+      if (hd < 0 || hd >= M.C) record_error(err, HSWA_ERR_BOUNDS, r, -4, hd);
+    }
+    for (int i = threadIdx.x; i < M.R; i += blockDim.x) {
+      const int pg = b.ring_table[(int64_t)r * M.R + i];
+      if (pg < 0 || pg >= num_pages) record_error(err, HSWA_ERR_BOUNDS, r, i, pg);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s) {
+  const int64_t total = (int64_t)p.total_q * 2 * p.m.Hkv * (p.m.D / 8);
+  if (total == 0) return cudaSuccess;
+  const int64_t blocks = (total + 255) / 256;
+  append_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,
+                                const int32_t* q_indptr, cudaStream_t s) {
+  if (B == 0) return cudaSuccess;
+  advance_kernel<<<(B + 127) / 128, 128, 0, s>>>(m, B, ctx_len, ring_head, q_indptr);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
+                                 int32_t* err, cudaStream_t s) {
+  if (b.B == 0) return cudaSuccess;
+  validate_kernel<<<b.B, 128, 0, s>>>(m, b, is_swa, num_pages, err);
+  return cudaGetLastError();
+}

@@ -1,0 +1,466 @@
+// Batched GQA decode attention over the hybrid KV cache (paper Sec. 2.2: decode is memory-bound, its cost is
+// the KV bytes read; Sec. 3.1.1: Full layers read pages through the block table, SWA layers read a ring of
+// R pages).  One thread block handles one (request, KV head, key split):
+//   - a producer warp walks the block table (or ring table) and streams 64-key K/V tiles into a multi-stage
+//     shared-memory ring with TMA tensor loads (128-byte swizzle), completion on mbarriers;
+//   - consumer warps each take whole tiles and keep an independent online-softmax state.  Scores are
+//     computed transposed on tensor cores, S^T[keys x heads] = K[keys x D] * Q^T[D x heads], so the 8 query
+//     heads of a GQA group are the N = 8 of m16n8k16 with no padding; P^T is moved into B-operand layout with
+//     movmatrix and O^T[D x heads] += V^T * P^T.  Row maxima are reduced with warp shuffles;
+//   - the block merges its warps' states and writes either the final output (one split) or a partial
+//     (m, l, o) for the combine kernel.
+// The new token's K/V row is patched into the staged tile and written to the cache by the block that owns
+// its position (fused append).
+#include "hswa_internal.cuh"
+
+namespace {
+using namespace hswa_dev;
+
+constexpr int TK = 64;  // keys per pipeline stage
+
+struct KeyRange {
+  int is_swa;
+  int span;   // Full: keys in this split; SWA: ring slots C
+  int head;   // SWA: ring head
+  int ctx;    // tokens cached before the step
+  int W, C;
+  // Is the key at index `idx` of this block's range visible to the query at position ctx?
+  __device__ __forceinline__ bool valid(int idx) const {
+    if (!is_swa) return idx < span;
+    if (idx >= C) return false;
+    int off = idx - head;
+    if (off < 0) off += C;
+    if (off == 0) return true;  // the new token itself
+    const int back = C - off;   // this slot holds position ctx - back
+    return back <= W - 1 && back <= ctx;
+  }
+};
+
+template <int D, int P, int NS, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, 2)
+decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
+  constexpr int HALVES = D / 64;
+  constexpr int PPT = TK / P;  // pages per tile
+  constexpr int HALF_BYTES = TK * 128;
+  constexpr int STAGE_BYTES = 2 * HALVES * HALF_BYTES;
+  constexpr int BOX_BYTES = P * 128;
+  constexpr int CHUNKS = D / 8;  // 16-byte chunks per row
+  constexpr int KS = D / 16;
+  static_assert(TK % P == 0, "page size must divide the tile");
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * NS];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+
+  const int r = blockIdx.x, split = blockIdx.y, kh = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const ModelParams& M = p.m;
+  const int ctx = p.b.ctx_len[r];
+  const int kv_len = ctx + 1;
+
+  KeyRange kr;
+  kr.is_swa = p.is_swa;
+  kr.ctx = ctx;
+  kr.W = M.W;
+  kr.C = M.C;
+  kr.head = 0;
+  int k_begin = 0;
+  if (!p.is_swa) {
+    k_begin = split * p.split_len;
+    if (k_begin >= kv_len) return;
+    kr.span = min(kv_len, k_begin + p.split_len) - k_begin;
+  } else {
+    if (split > 0) return;
+    kr.head = p.b.ring_head[r];
+    kr.span = M.C;
+  }
+  const int n_tiles = (kr.span + TK - 1) / TK;
+  const int idx_new = p.is_swa ? kr.head : ctx - k_begin;  // index of the new token in this block's range
+  const bool fuse = p.k_new != nullptr;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(smem_u32(&bars[i]), 1);       // full: producer's arrive + TMA bytes
+      mbar_init(smem_u32(&bars[NS + i]), 1);  // empty: one consumer warp per tile
+    }
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_pool);
+  }
+  __syncthreads();
+
+  // online-softmax state of a consumer warp (unused by the producer warp)
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+  float o[KS][4];
+#pragma unroll
+  for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  const int qd = (lane & 3) * 2;  // this thread's two heads: qd, qd + 1
+
+  if (warp == 0) {
+    // ---------------- producer ----------------
+    const int32_t* tbl;
+    int n_pages;
+    if (!p.is_swa) {
+      tbl = p.b.block_table + (int64_t)r * p.b.max_blocks + k_begin / P;
+      n_pages = (kr.span + P - 1) / P;
+    } else {
+      tbl = p.b.ring_table + (int64_t)r * M.R;
+      n_pages = M.R;
+    }
+    int pid_next = lane < n_pages ? tbl[lane] : 0;
+    int pid_cur = 0;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int pg0 = t * PPT;
+      if ((pg0 & 31) == 0) {
+        pid_cur = pid_next;
+        const int nx = pg0 + 32 + lane;
+        pid_next = nx < n_pages ? tbl[nx] : 0;
+      }
+      const int stage = t % NS;
+      if (t >= NS) {
+        if (!mbar_wait(smem_u32(&bars[NS + stage]), ((t / NS) - 1) & 1)) {
+          if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 1);
+          break;
+        }
+      }
+      uint32_t need = 0;
+      int pages[PPT];
+#pragma unroll
+      for (int i = 0; i < PPT; ++i) {
+        const int pgi = pg0 + i;
+        pages[i] = __shfl_sync(0xffffffffu, pid_cur, pgi & 31);
+        bool v = false;
+        if (pgi < n_pages)
+          for (int s = lane; s < P; s += 32) v |= kr.valid(pgi * P + s);
+        if (__any_sync(0xffffffffu, v)) need |= 1u << i;
+      }
+      if (lane == 0) {
+        uint32_t ok = 0;
+#pragma unroll
+        for (int i = 0; i < PPT; ++i) {
+          if (!(need & (1u << i))) continue;
+          if (pages[i] < 0 || pages[i] >= p.num_pages) {
+            record_error(p.err, HSWA_ERR_BOUNDS, r, pg0 + i, pages[i]);
+            continue;
+          }
+          ok |= 1u << i;
+        }
+        const uint32_t full_bar = smem_u32(&bars[stage]);
+        if (ok == 0) {
+          mbar_arrive(full_bar);
+        } else {
+          mbar_arrive_expect_tx(full_bar, __popc(ok) * 2 * HALVES * BOX_BYTES);
+          const uint32_t sbase = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int i = 0; i < PPT; ++i) {
+            if (!(ok & (1u << i))) continue;
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv)
+#pragma unroll
+              for (int hf = 0; hf < HALVES; ++hf)
+                tma_load_4d(sbase + (kv * HALVES + hf) * HALF_BYTES + i * BOX_BYTES, &tm_pool, full_bar, hf * 64, 0,
+                            kv * M.Hkv + kh, pages[i]);
+          }
+        }
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------- consumers ----------------
+    const int cw = warp - 1;
+    const int g_row = lane >> 2;  // head index used for the Q fragment (B operand column)
+    uint32_t qf[KS][2];
+    {
+      const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qf[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+        qf[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+      }
+    }
+    const int mi = lane >> 3, mr = lane & 7;
+    for (int t = cw; t < n_tiles; t += NW) {
+      const int stage = t % NS;
+      if (!mbar_wait(smem_u32(&bars[stage]), (t / NS) & 1)) {
+        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 2);
+        break;
+      }
+      uint8_t* sK = smem + stage * STAGE_BYTES;
+      uint8_t* sV = sK + HALVES * HALF_BYTES;
+      const uint32_t aK = smem_base + stage * STAGE_BYTES;
+      const uint32_t aV = aK + HALVES * HALF_BYTES;
+      const int tile_lo = t * TK;
+      bool wrote = false;
+
+      // fused append: patch the new token's row into the staged tile and write it to the cache
+      if (fuse && idx_new >= tile_lo && idx_new < tile_lo + TK) {
+        const int row = idx_new - tile_lo;
+        int page, slot;
+        if (!p.is_swa) {
+          page = p.b.block_table[(int64_t)r * p.b.max_blocks + ctx / P];
+          slot = ctx % P;
+        } else {
+          page = p.b.ring_table[(int64_t)r * M.R + kr.head / P];
+          slot = kr.head % P;
+        }
+        const bool page_ok = page >= 0 && page < p.num_pages;
+        if (!page_ok && lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, page);
+        for (int c = lane; c < 2 * CHUNKS; c += 32) {
+          const int kv = c / CHUNKS, ch = c % CHUNKS;
+          const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D + ch * 8;
+          const uint4 val = *reinterpret_cast<const uint4*>(src);
+          uint8_t* dst_s = (kv == 0 ? sK : sV) + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7);
+          *reinterpret_cast<uint4*>(dst_s) = val;
+          if (page_ok) {
+            __nv_bfloat16* dst_g = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * P + slot) * D + ch * 8;
+            *reinterpret_cast<uint4*>(dst_g) = val;
+          }
+        }
+        wrote = true;
+      }
+      // validity of the tile's 64 keys
+      const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
+      const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
+      if ((vm0 & vm1) != 0xffffffffu) {
+        // zero the V rows of invisible keys so that 0 * (stale or non-finite) cannot reach the output
+        for (int idx = lane; idx < TK * CHUNKS; idx += 32) {
+          const int row = idx / CHUNKS, ch = idx % CHUNKS;
+          const bool v = ((row < 32 ? vm0 : vm1) >> (row & 31)) & 1u;
+          if (!v) *reinterpret_cast<uint4*>(sV + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = make_uint4(0, 0, 0, 0);
+        }
+        wrote = true;
+      }
+      if (wrote) {
+        fence_proxy_async_smem();
+        __syncwarp();
+      }
+
+      if ((vm0 | vm1) != 0u) {
+        // S^T = K Q^T for the 64 keys (four 16-key blocks)
+        float s[4][4];
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          s[kb][0] = s[kb][1] = s[kb][2] = s[kb][3] = 0.f;
+          const int key = kb * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) {
+            const int chunk = 2 * ks + (mi >> 1);
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(aK + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+            mma_bf16_16816(s[kb], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
+          }
+        }
+        // mask, scale, tile maxima per head (this thread: heads qd and qd+1; keys lane/4 + 8j)
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const int keyA = kb * 16 + (lane >> 2), keyB = keyA + 8;
+          const bool vA = ((keyA < 32 ? vm0 : vm1) >> (keyA & 31)) & 1u;
+          const bool vB = ((keyB < 32 ? vm0 : vm1) >> (keyB & 31)) & 1u;
+          s[kb][0] = vA ? s[kb][0] * M.scale_log2 : -INFINITY;
+          s[kb][1] = vA ? s[kb][1] * M.scale_log2 : -INFINITY;
+          s[kb][2] = vB ? s[kb][2] * M.scale_log2 : -INFINITY;
+          s[kb][3] = vB ? s[kb][3] * M.scale_log2 : -INFINITY;
+          mx[0] = fmaxf(mx[0], fmaxf(s[kb][0], s[kb][2]));
+          mx[1] = fmaxf(mx[1], fmaxf(s[kb][1], s[kb][3]));
+        }
+#pragma unroll
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+          mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sh));
+          mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sh));
+        }
+        float m_use[2], alpha[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const float m_new = fmaxf(m_run[j], mx[j]);
+          m_use[j] = m_new == -INFINITY ? 0.f : m_new;
+          alpha[j] = fast_exp2(m_run[j] - m_use[j]);
+          m_run[j] = m_new;
+          l_run[j] *= alpha[j];
+        }
+#pragma unroll
+        for (int i = 0; i < KS; ++i) {
+          o[i][0] *= alpha[0];
+          o[i][1] *= alpha[1];
+          o[i][2] *= alpha[0];
+          o[i][3] *= alpha[1];
+        }
+        uint32_t pk[8];
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          pk[2 * kb] = pack_bf16x2(fast_exp2(s[kb][0] - m_use[0]), fast_exp2(s[kb][1] - m_use[1]));
+          pk[2 * kb + 1] = pack_bf16x2(fast_exp2(s[kb][2] - m_use[0]), fast_exp2(s[kb][3] - m_use[1]));
+          const float2 f0 = unpack_bf16x2(pk[2 * kb]), f1 = unpack_bf16x2(pk[2 * kb + 1]);
+          l_run[0] += f0.x + f1.x;  // sum the values the tensor core will actually multiply
+          l_run[1] += f0.y + f1.y;
+        }
+        // O^T += V^T P^T
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+          const uint32_t b0 = movmatrix_trans(pk[2 * kb]);
+          const uint32_t b1 = movmatrix_trans(pk[2 * kb + 1]);
+          const int key = kb * 16 + (mi >> 1) * 8 + mr;
+#pragma unroll
+          for (int mt = 0; mt < KS; ++mt) {
+            const int chunk = 2 * mt + (mi & 1);
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+            mma_bf16_16816(o[mt], a0, a1, a2, a3, b0, b1);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+    }
+
+    // per-warp row sums: lanes with equal (lane & 3) hold the same two heads
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+      l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+    }
+  }
+  __syncthreads();  // every tile has been consumed: the stage buffers can now hold the merge scratch
+  if (warp != 0) {
+    const int cw = warp - 1;
+    float* sc_o = reinterpret_cast<float*>(smem);  // [NW][8][D]
+    float* sc_ml = sc_o + NW * 8 * D;              // [NW][8][2]
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) {
+      const int d0 = mt * 16 + (lane >> 2);
+      sc_o[(cw * 8 + qd) * D + d0] = o[mt][0];
+      sc_o[(cw * 8 + qd + 1) * D + d0] = o[mt][1];
+      sc_o[(cw * 8 + qd) * D + d0 + 8] = o[mt][2];
+      sc_o[(cw * 8 + qd + 1) * D + d0 + 8] = o[mt][3];
+    }
+    if (lane < 4) {
+      sc_ml[(cw * 8 + qd) * 2 + 0] = m_run[0];
+      sc_ml[(cw * 8 + qd) * 2 + 1] = l_run[0];
+      sc_ml[(cw * 8 + qd + 1) * 2 + 0] = m_run[1];
+      sc_ml[(cw * 8 + qd + 1) * 2 + 1] = l_run[1];
+    }
+  }
+  __syncthreads();
+
+  // ---------------- merge the consumer warps' states ----------------
+  const float* sc_o = reinterpret_cast<const float*>(smem);
+  const float* sc_ml = sc_o + NW * 8 * D;
+  for (int idx = threadIdx.x; idx < M.G * D; idx += blockDim.x) {
+    const int g = idx / D, d = idx % D;
+    float mm = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sc_ml[(w * 8 + g) * 2]);
+    float L = 0.f, O = 0.f;
+    if (mm != -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const float f = fast_exp2(sc_ml[(w * 8 + g) * 2] - mm);
+        L += f * sc_ml[(w * 8 + g) * 2 + 1];
+        O += f * sc_o[(w * 8 + g) * D + d];
+      }
+    }
+    const int64_t row = (int64_t)r * M.Hq + kh * M.G + g;
+    if (p.max_splits == 1) {
+      const float val = L > 0.f ? O / L : 0.f;
+      if (M.out_fp32)
+        reinterpret_cast<float*>(p.out)[row * D + d] = val;
+      else
+        reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(val);
+      if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    } else {
+      p.part_o[(row * p.max_splits + split) * D + d] = O;
+      if (d == 0) p.part_ml[row * p.max_splits + split] = make_float2(mm, L);
+    }
+  }
+}
+
+// Merge split-K partials: out = sum_s 2^(m_s - m) o_s / sum_s 2^(m_s - m) l_s.  One warp per (request, head).
+template <int D>
+__global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
+  const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const ModelParams& M = p.m;
+  if (warp_global >= p.b.B * M.Hq) return;
+  const int r = warp_global / M.Hq;
+  const int64_t row = warp_global;
+  const int kv_len = p.b.ctx_len[r] + 1;
+  const int n_splits = min(p.max_splits, (kv_len + p.split_len - 1) / p.split_len);
+  const float2* ml = p.part_ml + row * p.max_splits;
+  const float* po = p.part_o + row * p.max_splits * D;
+  float mm = -INFINITY;
+  for (int s = lane; s < n_splits; s += 32) mm = fmaxf(mm, ml[s].x);
+#pragma unroll
+  for (int sh = 16; sh >= 1; sh >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, sh));
+  constexpr int PER = D / 32;
+  float acc[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+  float L = 0.f;
+  if (mm != -INFINITY) {
+    for (int s = 0; s < n_splits; ++s) {
+      const float2 v = ml[s];
+      const float f = fast_exp2(v.x - mm);
+      L += f * v.y;
+      if constexpr (PER == 4) {
+        const float4 x = *reinterpret_cast<const float4*>(po + (int64_t)s * D + lane * 4);
+        acc[0] += f * x.x;
+        acc[1] += f * x.y;
+        acc[2] += f * x.z;
+        acc[3] += f * x.w;
+      } else {
+        const float2 x = *reinterpret_cast<const float2*>(po + (int64_t)s * D + lane * 2);
+        acc[0] += f * x.x;
+        acc[1] += f * x.y;
+      }
+    }
+  }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) {
+    const float val = acc[i] * inv;
+    if (M.out_fp32)
+      reinterpret_cast<float*>(p.out)[row * D + lane * PER + i] = val;
+    else
+      reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + lane * PER + i] = __float2bfloat16_rn(val);
+  }
+  if (lane == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
+}
+
+template <int D, int P, int NS, int NW>
+cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, cudaStream_t s) {
+  constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
+  constexpr int SMEM = NS * STAGE_BYTES + 1024;
+  static_assert(NW * 8 * D * 4 + NW * 64 <= NS * STAGE_BYTES, "merge scratch must fit the stage buffers");
+  auto kern = decode_kernel<D, P, NS, NW>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  dim3 grid(p.b.B, p.max_splits, p.m.Hkv);
+  kern<<<grid, (NW + 1) * 32, SMEM, s>>>(tm, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t hswa_launch_decode(const hswa_handle*, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
+  if (p.b.B == 0) return cudaSuccess;
+  const int D = p.m.D, P = p.m.P;
+  if (D == 128 && P == 64) return launch_decode_t<128, 64, 3, 3>(tm_pool, p, s);
+  if (D == 128 && P == 32) return launch_decode_t<128, 32, 3, 3>(tm_pool, p, s);
+  if (D == 128 && P == 16) return launch_decode_t<128, 16, 3, 3>(tm_pool, p, s);
+  if (D == 64 && P == 64) return launch_decode_t<64, 64, 4, 3>(tm_pool, p, s);
+  if (D == 64 && P == 32) return launch_decode_t<64, 32, 4, 3>(tm_pool, p, s);
+  if (D == 64 && P == 16) return launch_decode_t<64, 16, 4, 3>(tm_pool, p, s);
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
+  const int rows = p.b.B * p.m.Hq;
+  if (rows == 0) return cudaSuccess;
+  const int blocks = (rows * 32 + 127) / 128;
+  if (p.m.D == 128)
+    combine_kernel<128><<<blocks, 128, 0, s>>>(p);
+  else
+    combine_kernel<64><<<blocks, 128, 0, s>>>(p);
+  return cudaGetLastError();
+}

@@ -1,0 +1,216 @@
+// Internal declarations shared by the library's translation units: handle, kernel parameter blocks and
+// the sm_100a device primitives (mbarrier, TMA, ldmatrix, mma) the kernels are written with.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hswa.h"
+
+typedef CUresult (*hswa_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                         const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                         CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                         CUtensorMapFloatOOBfill);
+
+struct hswa_handle {
+  hswa_config cfg;  // ring_pages and sm_scale resolved
+  int32_t ring_slots;  // C
+  int32_t group;       // G
+  int32_t device;
+  int32_t num_sms;
+  int32_t* err;  // device int32[4]
+  hswa_encode_tiled_fn encode_tiled;
+};
+
+// Model constants every kernel needs.
+struct ModelParams {
+  int32_t Hq, Hkv, G, D, P, W, R, C;
+  float scale_log2;  // sm_scale * log2(e)
+  int32_t out_fp32;
+};
+
+// The batch arrays as the kernels see them (device pointers).
+struct BatchParams {
+  int32_t B;
+  const int32_t* ctx_len;
+  const int32_t* q_indptr;
+  const int32_t* block_table;
+  int32_t max_blocks;
+  const int32_t* ring_table;
+  const int32_t* ring_head;
+};
+
+struct DecodeParams {
+  ModelParams m;
+  BatchParams b;
+  __nv_bfloat16* pool;
+  int64_t num_pages;
+  int32_t is_swa;
+  const __nv_bfloat16* q;      // [B][Hq][D]
+  const __nv_bfloat16* k_new;  // [B][Hkv][D] or null
+  const __nv_bfloat16* v_new;
+  void* out;   // [B][Hq][D]
+  float* lse;  // [B][Hq] or null
+  int32_t split_len;   // keys per split (multiple of 64)
+  int32_t max_splits;  // grid extent; 1 = write final output directly
+  float* part_o;       // [B*Hq][max_splits][D]
+  float2* part_ml;     // [B*Hq][max_splits] (m in log2 units, l)
+  int32_t* err;
+};
+
+struct AppendParams {
+  ModelParams m;
+  BatchParams b;
+  __nv_bfloat16* pool;
+  int64_t num_pages;
+  int32_t is_swa;
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  int32_t total_q;
+};
+
+struct PrefillParams {
+  ModelParams m;
+  BatchParams b;
+  __nv_bfloat16* pool;
+  int64_t num_pages;
+  int32_t is_swa;
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  void* out;
+  float* lse;
+  int32_t total_q;
+  int32_t max_q_len;
+  int32_t* err;
+};
+
+// Launchers implemented in the kernel translation units.
+cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s);
+cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s);
+cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
+cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
+cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,
+                                const int32_t* q_indptr, cudaStream_t s);
+cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
+                                 int32_t* err, cudaStream_t s);
+
+#ifdef __CUDACC__
+namespace hswa_dev {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void record_error(int32_t* err, int code, int a, int b, int c) {
+  if (atomicCAS(err, 0, code) == 0) {
+    err[1] = a;
+    err[2] = b;
+    err[3] = c;
+  }
+}
+
+// ---- mbarrier -----------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after about two seconds of SM clocks and reports false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (clock64() - t0 > 4000000000LL) return false;
+  }
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// ---- TMA (tiled tensor loads into shared memory, completion on an mbarrier) ---------------------------
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
+
+// ---- warp-level matrix primitives ---------------------------------------------------------------------
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float2 unpack_bf16x2(uint32_t u) {
+  __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&u);
+  return __bfloat1622float2(v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a tile of 128-byte rows written by TMA
+// with the 128-byte swizzle (the tile base is 1024-byte aligned).
+__device__ __forceinline__ uint32_t swz128(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+__device__ __forceinline__ int math_mod(int a, int m) {
+  int r = a % m;
+  return r < 0 ? r + m : r;
+}
+
+}  // namespace hswa_dev
+#endif  // __CUDACC__

@@ -1,0 +1,343 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the same seeded
+inputs.  Indexing and pool bytes must match bit for bit; attention outputs (fp32 output mode) within
+1e-2 max abs error (bf16 inputs, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hswa_oracle as orc
+from paper_2607_13095_b200 import binding as hb
+from paper_2607_13095_b200 import workloads as wl
+from helpers import build_scenario
+from gpu_utils import dev_batch, dev_i32, make_handle, to_dev_bf16, to_host_bits, workspace_for
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def dims(G, D, P, Hkv=2, W=128):
+    return wl.Dims(num_q_heads=G * Hkv, num_kv_heads=Hkv, head_dim=D, page_size=P, window=W)
+
+
+def check_no_async_error(h):
+    st = hb.hswa_get_async_error(h)
+    assert st[0] == hb.HSWA_OK, st
+
+
+# ---------------------------------------------------------------------------------------------------------
+def run_append(sc, is_swa, decode):
+    h = make_handle(sc.dims)
+    pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+    layer = hb.Layer(pool, is_swa)
+    hb.hswa_validate_batch(h, layer, dev_batch(sc.tables, decode))
+    hb.hswa_kv_append(h, layer, dev_batch(sc.tables, decode), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new))
+    check_no_async_error(h)
+    ol = sc.layer(is_swa)
+    orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+    got = to_host_bits(pool)
+    assert np.array_equal(got, ol.pool), "pool bytes differ after append"
+
+
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_append_config1(is_swa):
+    for kind in ("decode", "prefill"):
+        w = wl.config1(kind)
+        sc = build_scenario(w.dims, w.tables.ctx_len, w.tables.q_len, seed=1, scale=w.value_scale, ring_keep=w.dims.ring_slots)
+        run_append(sc, is_swa, decode=False)
+        if kind == "decode":
+            run_append(sc, is_swa, decode=True)
+
+
+@pytest.mark.parametrize("d", [dims(4, 64, 16, 1), dims(8, 128, 64), dims(2, 128, 32, 3)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_append_sweep(d, is_swa):
+    C, P = d.ring_slots, d.page_size
+    ctx = [0, 1, P - 1, P, C - 1, C + 1, 3 * C + 5, 700]
+    q_len = [2 * C + 3, 1, C, 17, 0, C + 1, 65, 300]
+    sc = build_scenario(d, ctx, q_len, seed=5, ring_keep=C)
+    run_append(sc, is_swa, decode=False)
+
+
+# ---------------------------------------------------------------------------------------------------------
+def run_decode(sc, is_swa, fused, out_dtype=torch.float32, check_pool=True):
+    d, t = sc.dims, sc.tables
+    h = make_handle(d, out_dtype, sc.cfg.sm_scale)
+    pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+    layer = hb.Layer(pool, is_swa)
+    b = dev_batch(t, decode=True)
+    q, k_new, v_new = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    out = torch.full((t.batch, d.num_q_heads, d.head_dim), float("nan"), dtype=out_dtype, device="cuda")
+    lse = torch.full((t.batch, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    ws = workspace_for(h, t)
+    if fused:
+        hb.hswa_decode_attn(h, layer, b, q, k_new, v_new, out, lse, ws)
+    else:
+        hb.hswa_kv_append(h, layer, b, k_new, v_new)
+        hb.hswa_decode_attn(h, layer, b, q, None, None, out, lse, ws)
+    check_no_async_error(h)
+    ol = sc.layer(is_swa)
+    ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+    got = out.float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - ref).max() if t.batch else 0.0
+    lerr = np.abs(lse.cpu().numpy() - ref_lse).max() if t.batch else 0.0
+    assert np.isfinite(got).all()
+    if check_pool:
+        orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+        assert np.array_equal(to_host_bits(pool), ol.pool), "pool bytes differ after fused append"
+    return err, lerr
+
+
+@pytest.mark.parametrize("is_swa", [False, True])
+@pytest.mark.parametrize("fused", [True, False])
+def test_decode_config1(is_swa, fused):
+    w = wl.config1("decode")
+    sc = build_scenario(w.dims, w.tables.ctx_len, w.tables.q_len, seed=1, scale=w.value_scale)
+    err, lerr = run_decode(sc, is_swa, fused)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+@pytest.mark.parametrize("d", [dims(4, 64, 16, 1), dims(8, 128, 64), dims(1, 128, 64, 3), dims(3, 64, 32),
+                               dims(8, 128, 16), dims(5, 64, 64)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_decode_sweep(d, is_swa):
+    W, P, C = d.window, d.page_size, d.ring_slots
+    ctx = sorted({0, 1, 2, 62, 63, 64, 65, W - 2, W - 1, W, W + 1, P - 1, P, P + 1, C - 1, C, C + 1, 3 * C + 5,
+                  255, 256, 257, 2047, 2048, 2049, 5000})
+    sc = build_scenario(d, ctx, [1] * len(ctx), seed=7)
+    for fused in (True, False):
+        err, lerr = run_decode(sc, is_swa, fused)
+        assert err <= TOL and lerr <= TOL, (fused, err, lerr)
+
+
+def test_decode_long_split_and_bf16_out():
+    d = dims(8, 128, 64, 2)
+    sc = build_scenario(d, [40000, 9000, 33, 20481], [1, 1, 1, 1], seed=9)
+    err, lerr = run_decode(sc, False, True)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+    err, _ = run_decode(sc, False, True, out_dtype=torch.bfloat16)
+    assert err <= TOL, err
+    err, _ = run_decode(sc, True, True, out_dtype=torch.bfloat16)
+    assert err <= TOL, err
+
+
+def test_decode_large_values_and_shared_prefix():
+    d = dims(8, 128, 64, 2)
+    sc = build_scenario(d, [64 * 5 + 3, 64 * 5 + 100, 64 * 9], [1, 1, 1], seed=10, shared_prefix_tokens=64 * 5)
+    assert (sc.tables.block_table[:, :5] == sc.tables.block_table[0, :5]).all()
+    for is_swa in (False, True):
+        err, lerr = run_decode(sc, is_swa, True)
+        assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+def test_decode_page_permutation_bit_identical():
+    d = dims(8, 128, 64, 2)
+    outs = []
+    for permute in (True, False):
+        sc = build_scenario(d, [5000, 300, 2049], [1, 1, 1], seed=11, permute=permute,
+                            ring_head=np.array([5, 100, 191]))
+        h = make_handle(d)
+        t = sc.tables
+        res = []
+        for is_swa in (False, True):
+            layer = hb.Layer(to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool), is_swa)
+            out = torch.zeros((t.batch, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+            hb.hswa_decode_attn(h, layer, dev_batch(t, True), to_dev_bf16(sc.q), to_dev_bf16(sc.k_new),
+                                to_dev_bf16(sc.v_new), out, None, workspace_for(h, t))
+            res.append(out.cpu())
+        outs.append(res)
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+# ---------------------------------------------------------------------------------------------------------
+def run_prefill(sc, is_swa, fuse_append=True, out_dtype=torch.float32):
+    d, t = sc.dims, sc.tables
+    h = make_handle(d, out_dtype, sc.cfg.sm_scale)
+    pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+    layer = hb.Layer(pool, is_swa)
+    b = dev_batch(t, decode=False)
+    q, k_new, v_new = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    out = torch.full((t.total_q, d.num_q_heads, d.head_dim), float("nan"), dtype=out_dtype, device="cuda")
+    lse = torch.full((t.total_q, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    hb.hswa_prefill_attn(h, layer, b, q, k_new, v_new, fuse_append, out, lse, workspace_for(h, t))
+    check_no_async_error(h)
+    ol = sc.layer(is_swa)
+    ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    if fuse_append:
+        orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+    assert np.array_equal(to_host_bits(pool), ol.pool), "pool bytes differ after prefill"
+    return np.abs(got - ref).max(), np.abs(lse.cpu().numpy() - ref_lse).max()
+
+
+@pytest.mark.parametrize("is_swa", [False, True])
+@pytest.mark.parametrize("fuse_append", [True, False])
+def test_prefill_config1(is_swa, fuse_append):
+    w = wl.config1("prefill")
+    sc = build_scenario(w.dims, w.tables.ctx_len, w.tables.q_len, seed=1, scale=w.value_scale)
+    err, lerr = run_prefill(sc, is_swa, fuse_append)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+@pytest.mark.parametrize("d", [dims(4, 64, 16, 1), dims(8, 128, 64), dims(2, 128, 32, 3), dims(1, 64, 64)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_prefill_sweep(d, is_swa):
+    C, P, W = d.ring_slots, d.page_size, d.window
+    ctx = [0, 1, W - 1, W, P + 1, C - 1, 3 * C + 5, 700, 0, 130]
+    q_len = [2 * C + 3, 1, 64, 65, 17, C + 1, 66, 300, 129, 0]
+    sc = build_scenario(d, ctx, q_len, seed=13)
+    err, lerr = run_prefill(sc, is_swa)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+def test_prefill_wrong_order_on_ring_is_detected():
+    """Contract guard: appending a long chunk to a ring BEFORE attending loses keys the chunk's first queries
+    need, so the library's attend-then-append order is the only valid one on SWA layers."""
+    d = dims(4, 64, 16, 1)
+    sc = build_scenario(d, [512], [64], seed=14, ring_keep=d.ring_slots)
+    t = sc.tables
+    h = make_handle(d)
+    pool = to_dev_bf16(sc.swa_pool)
+    layer = hb.Layer(pool, True)
+    b = dev_batch(t, decode=False)
+    q, k_new, v_new = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    hb.hswa_kv_append(h, layer, b, k_new, v_new)          # wrong: append first
+    out = torch.zeros((t.total_q, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    hb.hswa_prefill_attn(h, layer, b, q, k_new, v_new, False, out, None, None)
+    ref, _ = orc.attention(sc.cfg, sc.layer(True), sc.batch(), sc.q, sc.k_new, sc.v_new)
+    assert np.abs(out.cpu().numpy() - ref).max() > TOL
+
+
+# ---------------------------------------------------------------------------------------------------------
+def test_step_advance_matches_oracle():
+    d = dims(8, 128, 64)
+    t = wl.make_tables(d, [0, 5, 1000, 191], [1, 200, 64, 7], seed=3)
+    h = make_handle(d)
+    for q_indptr in (t.q_indptr, None):
+        ctx, head = dev_i32(t.ctx_len), dev_i32(t.ring_head)
+        hb.hswa_step_advance(h, t.batch, ctx, head, None if q_indptr is None else dev_i32(q_indptr))
+        ectx, ehead = t.ctx_len.copy(), t.ring_head.copy()
+        orc.step_advance(orc.OracleConfig(d.num_q_heads, d.num_kv_heads, d.head_dim, d.page_size), ectx, ehead, q_indptr)
+        assert np.array_equal(ctx.cpu().numpy(), ectx) and np.array_equal(head.cpu().numpy(), ehead)
+
+
+def test_multi_step_decode_history():
+    """Prefill a prompt, then decode several tokens with fused append and step advance; every step must match
+    the oracle run on the same evolving state (ring wraps included)."""
+    d = dims(4, 64, 16, 1)
+    sc = build_scenario(d, [0, 37], [150, 120], seed=15)
+    t = sc.tables
+    h = make_handle(d)
+    steps = 40
+    big_t = wl.make_tables(d, [0, 37], [150 + steps, 120 + steps], seed=15, ring_head=t.ring_head)
+    # device state (block table sized for the whole history)
+    pools = {False: to_dev_bf16(np.resize(sc.full_pool, (big_t.num_full_pages,) + sc.full_pool.shape[1:])),
+             True: to_dev_bf16(sc.swa_pool)}
+    o_pools = {False: np.resize(sc.full_pool, (big_t.num_full_pages,) + sc.full_pool.shape[1:]).copy(),
+               True: sc.swa_pool.copy()}
+    # history already present in sc pools was placed with sc.tables' block table: rebuild with big_t instead
+    sc2 = build_scenario(d, [0, 37], [150, 120], seed=15, ring_head=t.ring_head)
+    bt = big_t.block_table
+    ctx = dev_i32(t.ctx_len)
+    head = dev_i32(t.ring_head)
+    octx, ohead = t.ctx_len.copy(), t.ring_head.copy()
+    # place the 37-token history of request 1 through the library itself (append on both layers)
+    hist_b = hb.Batch(dev_i32([0, 0]), dev_i32(bt), dev_i32(big_t.ring_table), dev_i32(np.mod(t.ring_head - t.ctx_len, d.ring_slots)),
+                      dev_i32([0, 0, 37]), max_q_len=37, total_q=37, max_ctx_len=0)
+    hk, hv = sc2.k_seq[1][:37], sc2.v_seq[1][:37]
+    ohist = orc.OracleBatch(np.zeros(2, np.int32), bt, big_t.ring_table, np.mod(t.ring_head - t.ctx_len, d.ring_slots),
+                            np.array([0, 0, 37], np.int32))
+    for is_swa in (False, True):
+        pools[is_swa].view(torch.int16).fill_(0)
+        o_pools[is_swa][:] = 0
+        hb.hswa_kv_append(h, hb.Layer(pools[is_swa], is_swa), hist_b, to_dev_bf16(hk), to_dev_bf16(hv))
+        orc.kv_append(sc2.cfg, orc.OracleLayer(o_pools[is_swa], is_swa), ohist, hk, hv)
+    # step 0: prefill
+    qi = t.q_indptr
+    for step in range(steps + 1):
+        if step == 0:
+            q_bits, k_bits, v_bits, q_indptr = sc2.q, sc2.k_new, sc2.v_new, qi
+        else:
+            q_bits = wl.bf16_bits_normal(1000 + step, (2, d.num_q_heads, d.head_dim))
+            k_bits = wl.bf16_bits_normal(2000 + step, (2, d.num_kv_heads, d.head_dim))
+            v_bits = wl.bf16_bits_normal(3000 + step, (2, d.num_kv_heads, d.head_dim))
+            q_indptr = None
+        T = q_bits.shape[0]
+        ob = orc.OracleBatch(octx.copy(), bt, big_t.ring_table, ohead.copy(), q_indptr)
+        gb = hb.Batch(ctx, dev_i32(bt), dev_i32(big_t.ring_table), head, None if q_indptr is None else dev_i32(q_indptr),
+                      max_q_len=150 if step == 0 else 1, total_q=T, max_ctx_len=int(octx.max()))
+        for is_swa in (False, True):
+            layer = hb.Layer(pools[is_swa], is_swa)
+            out = torch.zeros((T, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+            ws = torch.empty(hb.hswa_workspace_bytes(h, 2, T, 400) + 256, dtype=torch.uint8, device="cuda")
+            if step == 0:
+                hb.hswa_prefill_attn(h, layer, gb, to_dev_bf16(q_bits), to_dev_bf16(k_bits), to_dev_bf16(v_bits), True, out, None, ws)
+            else:
+                hb.hswa_decode_attn(h, layer, gb, to_dev_bf16(q_bits), to_dev_bf16(k_bits), to_dev_bf16(v_bits), out, None, ws)
+            ol = orc.OracleLayer(o_pools[is_swa], is_swa)
+            ref, _ = orc.attention(sc2.cfg, ol, ob, q_bits, k_bits, v_bits)
+            orc.kv_append(sc2.cfg, ol, ob, k_bits, v_bits)
+            assert np.abs(out.cpu().numpy() - ref).max() <= TOL, (step, is_swa)
+            assert np.array_equal(to_host_bits(pools[is_swa]), o_pools[is_swa]), (step, is_swa)
+        hb.hswa_step_advance(h, 2, ctx, head, None if q_indptr is None else dev_i32(q_indptr))
+        orc.step_advance(sc2.cfg, octx, ohead, q_indptr)
+        assert np.array_equal(ctx.cpu().numpy(), octx) and np.array_equal(head.cpu().numpy(), ohead)
+    check_no_async_error(h)
+
+
+# ---------------------------------------------------------------------------------------------------------
+def test_validate_batch_reports_bad_ids():
+    d = dims(8, 128, 64)
+    sc = build_scenario(d, [300, 70], [1, 1], seed=16)
+    t = sc.tables
+    h = make_handle(d)
+    full = hb.Layer(to_dev_bf16(sc.full_pool), False)
+    swa = hb.Layer(to_dev_bf16(sc.swa_pool), True)
+    hb.hswa_validate_batch(h, full, dev_batch(t, True))
+    hb.hswa_validate_batch(h, swa, dev_batch(t, True))
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    # corrupt the HOST copy of the block table, then validate: the error word names request and entry
+    bad = t.block_table.copy()
+    bad[1, 0] = t.num_full_pages + 7
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(bad), dev_i32(t.ring_table), dev_i32(t.ring_head), max_ctx_len=300)
+    hb.hswa_validate_batch(h, full, b)
+    st = hb.hswa_get_async_error(h)
+    assert st == (hb.HSWA_ERR_BOUNDS, 1, 0, t.num_full_pages + 7), st
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK  # cleared
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32([0, d.ring_slots]), max_ctx_len=300)
+    hb.hswa_validate_batch(h, swa, b)
+    st = hb.hswa_get_async_error(h)
+    assert st[0] == hb.HSWA_ERR_BOUNDS and st[1] == 1, st
+    # a decode over the corrupted table skips the bad page, records the error and returns
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(bad), dev_i32(t.ring_table), dev_i32(t.ring_head), max_ctx_len=300)
+    out = torch.zeros((2, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    hb.hswa_decode_attn(h, full, b, to_dev_bf16(sc.q), None, None, out, None, workspace_for(h, t))
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_ERR_BOUNDS
+
+
+def test_host_side_argument_errors():
+    d = dims(8, 128, 64)
+    sc = build_scenario(d, [5000, 70], [1, 1], seed=17)
+    t = sc.tables
+    h = make_handle(d)
+    full = hb.Layer(to_dev_bf16(sc.full_pool), False)
+    b = dev_batch(t, True)
+    q = to_dev_bf16(sc.q)
+    out = torch.zeros((2, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn(h, full, b, q, None, None, out, None, None)   # split-K needs a workspace
+    assert e.value.status == hb.HSWA_ERR_WORKSPACE
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn(h, full, b, q, to_dev_bf16(sc.k_new), None, out, None, workspace_for(h, t))
+    assert e.value.status == hb.HSWA_ERR_INVALID_ARG
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn(h, full, dev_batch(t, False), q, None, None, out, None, workspace_for(h, t))
+    assert e.value.status == hb.HSWA_ERR_INVALID_ARG                     # decode takes no q_indptr
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_prefill_attn(h, full, dev_batch(t, False), q, None, None, True, out)
+    assert e.value.status == hb.HSWA_ERR_INVALID_ARG                     # prefill needs k_new / v_new
+    # empty batch is a no-op
+    empty = hb.Batch(dev_i32(np.zeros(0)), dev_i32(np.zeros((0, 1))), dev_i32(np.zeros((0, 3))), dev_i32(np.zeros(0)),
+                     max_q_len=1, total_q=0)
+    hb.hswa_decode_attn(h, full, empty, q, None, None, out, None, None)
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
