@@ -132,6 +132,27 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
                              const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, void* stream);
 
+/* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart of this
+ * call; it exists for deployment reasons only.)
+ * Same arguments, results and errors as hswa_decode_attn, minus the workspace: the split-K partials go to a
+ * fixed array of HSWA_STATIC_WS_BYTES bytes that is part of the library's device image, so this call performs
+ * no cudaMalloc / cudaFree and calls no allocating routine.  It serves code that runs under a fixed memory
+ * budget, or inside a section where an allocation (and the device-wide synchronisation it implies) is not
+ * allowed, and that therefore has no workspace to offer.
+ *   - Limit: a batch whose partials need more than HSWA_STATIC_WS_BYTES (roughly B * Hq * ceil((max_ctx_len
+ *     + 1) / 2048) * (4 * D + 8) bytes on a Full layer; SWA layers need none) is rejected with
+ *     HSWA_ERR_WORKSPACE and nothing is launched.
+ *   - Every GPU that loads the library holds the array until the process exits.
+ *   - The first call on a device looks up the array's device address (with that device current, which must be
+ *     the handle's device); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps whatever the last call left there.  No part of
+ *     it has to start at zero: each call writes every partial it later reads.  Two calls that overlap on the
+ *     GPU (different streams, or different handles) race on it; issue them on one stream. */
+#define HSWA_STATIC_WS_BYTES (64u << 20)
+hswa_status hswa_decode_attn_static_ws(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch,
+                                       const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                                       void* stream);
+
 /* Chunked prefill attention: request r extends its cached context by n[r] new tokens.
  * q: device bf16 [T][Hq][D]; k_new, v_new: device bf16 [T][Hkv][D] (required); out: device [T][Hq][D];
  * lse: device fp32 [T][Hq] or NULL.

@@ -24,7 +24,7 @@ HSWA_ERR_TIMEOUT = 6
 
 EXPORTS = [
     "hswa_create", "hswa_destroy", "hswa_workspace_bytes", "hswa_validate_batch", "hswa_kv_append",
-    "hswa_decode_attn", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
+    "hswa_decode_attn", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
 ]
 
 
@@ -83,6 +83,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_kv_append.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp]
     lib.hswa_decode_attn.restype = C.c_int
     lib.hswa_decode_attn.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.hswa_decode_attn_static_ws.restype = C.c_int
+    lib.hswa_decode_attn_static_ws.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp, vp, vp, vp]
     lib.hswa_prefill_attn.restype = C.c_int
     lib.hswa_prefill_attn.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp, i32, vp, vp, vp,
                                       sz, vp]
@@ -190,6 +192,18 @@ def hswa_decode_attn(h: Handle, layer: Layer, batch: Batch, q, k_new, v_new, out
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().hswa_decode_attn(h.ptr, C.byref(layer.c), C.byref(batch.c), _ptr(q), _ptr(k_new), _ptr(v_new),
                                    _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes, _stream()), "hswa_decode_attn")
+
+
+STATIC_WS_BYTES = 64 << 20
+
+
+def hswa_decode_attn_static_ws(h: Handle, layer: Layer, batch: Batch, q, k_new, v_new, out, lse=None):
+    """Decode attention for callers that cannot allocate: the split-K scratch is a fixed STATIC_WS_BYTES array
+    inside the library (shared by all calls on the device, so keep them on one stream).  Make the first call
+    on a device outside any stream capture."""
+    _check(load().hswa_decode_attn_static_ws(h.ptr, C.byref(layer.c), C.byref(batch.c), _ptr(q), _ptr(k_new),
+                                             _ptr(v_new), _ptr(out), _ptr(lse), _stream()),
+           "hswa_decode_attn_static_ws")
 
 
 def hswa_prefill_attn(h: Handle, layer: Layer, batch: Batch, q, k_new, v_new, fuse_append, out, lse=None,
