@@ -88,6 +88,19 @@ hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtenso
   return rc == CUDA_SUCCESS ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
+// 3-D view of a [T][heads][D] activation tensor for TMA: box {64, 1, box_rows}, 128-byte swizzle.
+hswa_status make_rows_map(const hswa_handle* h, const void* ptr, int heads, int64_t rows, int box_rows, CUtensorMap* tm) {
+  const cuuint64_t D = (cuuint64_t)h->cfg.head_dim;
+  cuuint64_t dims[3] = {D, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {D * 2, D * 2 * (cuuint64_t)heads};
+  cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult rc = h->encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -279,7 +292,18 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
   p.total_q = b->total_q;
   p.max_q_len = b->max_q_len;
   p.err = h->err;
-  if (hswa_launch_prefill_mma(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  const int64_t tc_tiles = (int64_t)b->batch * ((b->max_q_len + 127) / 128);
+  if (hswa_prefill_tc_supported(p.m) && b->q_indptr != nullptr && tc_tiles <= 65535) {
+    // tcgen05 / TMEM / TMA tile kernel
+    CUtensorMap tm_pool, tm_q, tm_k, tm_v;
+    if ((st = make_pool_map(h, layer, &tm_pool)) != HSWA_OK) return st;
+    if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->total_q, 128, &tm_q)) != HSWA_OK) return st;
+    if ((st = make_rows_map(h, k_new, h->cfg.num_kv_heads, b->total_q, 128, &tm_k)) != HSWA_OK) return st;
+    if ((st = make_rows_map(h, v_new, h->cfg.num_kv_heads, b->total_q, 128, &tm_v)) != HSWA_OK) return st;
+    if (hswa_launch_prefill_tc(tm_pool, tm_q, tm_k, tm_v, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  } else {
+    if (hswa_launch_prefill_mma(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  }
   if (fuse_append) {
     // stream order puts the append after every read of the pre-append ring contents
     AppendParams a;

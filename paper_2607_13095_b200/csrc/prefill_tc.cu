@@ -1,0 +1,480 @@
+// Chunked prefill attention on 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM, operands
+// staged by TMA) for head_dim 128, page size 64 and an even GQA group.  Paper Sec. 2.1: prefill is
+// compute-bound, Full layers attend to the whole prefix, SWA layers only inside the window; Sec. 3.1.1: Full
+// layers read pages through the block table, SWA layers a ring (as it is before this chunk's append).
+//
+// One thread block = 128 query tokens x 2 query heads of one GQA group (two 128-row Q tiles that share every
+// K/V tile and every mask).  Warp roles:
+//   warps 0-3   softmax for Q tile 0 (one thread per row: TMEM lane = row, so row max / row sum are thread-local)
+//   warps 4-7   softmax for Q tile 1
+//   warp  8     TMA producer: Q once, then 128-key K and V tiles through two 2-stage rings
+//   warp  9     MMA issuer: S_i = Q_i K^T (SS form), O_i += P_i V (TS form, P read from TMEM where it
+//               overwrites S_i), in the order PV0(j), S0(j+1), PV1(j), S1(j+1) so that one tile's softmax
+//               overlaps the other tile's MMAs
+// TMEM columns: S0 0-127, S1 128-255, O0 256-383, O1 384-511 (all fp32; P_i = bf16 pairs in the first 64
+// columns of S_i).  O is rescaled lazily: only when a row maximum grows by more than 2^8.
+//
+// Key tiles: phase A covers cached positions (Full: pages 2a, 2a+1 of the block table; SWA: the ring pages,
+// only for the first tokens of the chunk), phase B covers the chunk's own K/V in chunk-relative 128-token
+// tiles, so every tile has a single source and masks take care of ragged edges.  Tiles wholly above the
+// diagonal or wholly below the window are never loaded or multiplied.
+#include "hswa_internal.cuh"
+
+namespace {
+using namespace hswa_dev;
+
+constexpr int BM = 128;               // query rows per Q tile
+constexpr int BN = 128;               // keys per tile
+constexpr int HD = 128;               // head dim
+constexpr int PG = 64;                // page size
+constexpr int HALF_BYTES = 128 * 128; // [128 rows][128 B]: one 64-element half of a 128-row tile
+constexpr int TILE_BYTES = 2 * HALF_BYTES;
+constexpr int KV_STAGES = 2;
+constexpr int NUM_THREADS = 320;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int OFF_Q = 0;                                  // 2 Q tiles
+constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;             // KV_STAGES K tiles
+constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;     // KV_STAGES V tiles
+constexpr int SMEM_TILES = OFF_V + KV_STAGES * TILE_BYTES;  // 196608
+constexpr int SMEM_BYTES = SMEM_TILES + 1024;
+
+constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [key][d] with d contiguous
+
+// barrier indices
+enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PFULL = 11,
+       BAR_OFINAL = 13, NUM_BARS = 14 };
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
+      "}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(0u)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t"
+      "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc), "r"(0u)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version for this architecture
+  d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(addr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};" ::"r"(r[0]),
+      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
+      "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]),
+      "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(addr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};" ::"r"(r[0]),
+      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(addr)
+      : "memory");
+}
+
+// The sequence of key tiles one block walks: nA cached tiles, then chunk tiles c_lo .. c_lo + nB - 1.
+struct TileSeq {
+  int nA, c_lo, nB;
+  __device__ __forceinline__ int total() const { return nA + nB; }
+};
+__device__ __forceinline__ TileSeq tile_seq(int is_swa, int ctx, int b, int W, int R) {
+  TileSeq s;
+  if (!is_swa) {
+    s.nA = (ctx + BN - 1) / BN;
+    s.c_lo = 0;
+  } else {
+    const bool ring = ctx > 0 && b * BM < W - 1;  // some row of this tile reaches below the chunk
+    s.nA = ring ? (R + 1) / 2 : 0;
+    const int low = b * BM - W + 1;  // lowest chunk-relative key any row needs
+    s.c_lo = low > 0 ? low / BN : 0;
+  }
+  s.nB = b - s.c_lo + 1;
+  return s;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_constant__ CUtensorMap tm_q,
+                  const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                  const PrefillParams p, const int max_tiles) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[NUM_BARS];
+  __shared__ uint32_t tmem_base_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const ModelParams& M = p.m;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pair = blockIdx.x, kh = blockIdx.y;
+  const int r = blockIdx.z % p.b.B;
+  const int b = max_tiles - 1 - (int)(blockIdx.z / p.b.B);  // longest tiles are scheduled first
+  const int t0 = p.b.q_indptr[r];
+  const int n = p.b.q_indptr[r + 1] - t0;
+  if (b * BM >= n) return;  // uniform for the block
+  if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;  // an earlier block gave up: do not queue behind it
+  const int ctx = p.b.ctx_len[r];
+  const int head = p.is_swa ? p.b.ring_head[r] : 0;
+  const int h0 = kh * M.G + pair * 2;
+  const TileSeq seq = tile_seq(p.is_swa, ctx, b, M.W, M.R);
+  const int n_tiles = seq.total();
+
+  auto bar = [&](int i) { return smem_u32(&bars[i]); };
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(BAR_Q), 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(bar(BAR_KFULL + s), 1);
+      mbar_init(bar(BAR_KEMPTY + s), 1);
+      mbar_init(bar(BAR_VFULL + s), 1);
+      mbar_init(bar(BAR_VEMPTY + s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_SFULL + i), 1);
+      mbar_init(bar(BAR_PFULL + i), 128);
+    }
+    mbar_init(bar(BAR_OFINAL), 1);
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+
+  if (warp == 8) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_pool);
+      tma_prefetch_desc(&tm_q);
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_v);
+      mbar_arrive_expect_tx(bar(BAR_Q), 2 * TILE_BYTES);
+      for (int i = 0; i < 2; ++i)
+        for (int hf = 0; hf < 2; ++hf)
+          tma_load_3d(sbase + OFF_Q + i * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(BAR_Q), hf * 64, h0 + i, t0 + b * BM);
+    }
+    // page ids of the cached tiles, 32 at a time
+    const int32_t* tbl = p.is_swa ? p.b.ring_table + (int64_t)r * M.R : p.b.block_table + (int64_t)r * p.b.max_blocks;
+    const int n_pages = p.is_swa ? M.R : (ctx + PG - 1) / PG;
+    int pid_next = lane < n_pages ? tbl[lane] : 0;
+    int pid_cur = 0;
+    bool ok = true;
+    for (int j = 0; j < n_tiles && ok; ++j) {
+      const int stage = j % KV_STAGES;
+      int pg[2] = {0, 0};
+      if (j < seq.nA) {
+        if (((2 * j) & 31) == 0) {
+          pid_cur = pid_next;
+          const int nx = 2 * j + 32 + lane;
+          pid_next = nx < n_pages ? tbl[nx] : 0;
+        }
+        const int i0 = 2 * j, i1 = (2 * j + 1 < n_pages) ? 2 * j + 1 : 2 * j;  // a missing page repeats its neighbour
+        pg[0] = __shfl_sync(0xffffffffu, pid_cur, i0 & 31);
+        pg[1] = __shfl_sync(0xffffffffu, pid_cur, i1 & 31);
+      }
+      if (lane == 0) {
+        if (j >= KV_STAGES) {
+          const uint32_t par = ((j / KV_STAGES) - 1) & 1;
+          if (!mbar_wait(bar(BAR_KEMPTY + stage), par) || !mbar_wait(bar(BAR_VEMPTY + stage), par)) {
+            record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 10);
+            ok = false;
+          }
+        }
+        if (ok) {
+          const uint32_t dK = sbase + OFF_K + stage * TILE_BYTES, dV = sbase + OFF_V + stage * TILE_BYTES;
+          mbar_arrive_expect_tx(bar(BAR_KFULL + stage), TILE_BYTES);
+          mbar_arrive_expect_tx(bar(BAR_VFULL + stage), TILE_BYTES);
+          if (j < seq.nA) {
+            for (int q = 0; q < 2; ++q) {
+              int page = pg[q];
+              if (page < 0 || page >= p.num_pages) {
+                record_error(p.err, HSWA_ERR_BOUNDS, r, 2 * j + q, page);
+                page = 0;
+              }
+              for (int hf = 0; hf < 2; ++hf) {
+                tma_load_4d(dK + hf * HALF_BYTES + q * PG * 128, &tm_pool, bar(BAR_KFULL + stage), hf * 64, 0, kh, page);
+                tma_load_4d(dV + hf * HALF_BYTES + q * PG * 128, &tm_pool, bar(BAR_VFULL + stage), hf * 64, 0,
+                            M.Hkv + kh, page);
+              }
+            }
+          } else {
+            const int tok = t0 + (seq.c_lo + (j - seq.nA)) * BN;
+            for (int hf = 0; hf < 2; ++hf) {
+              tma_load_3d(dK + hf * HALF_BYTES, &tm_k, bar(BAR_KFULL + stage), hf * 64, kh, tok);
+              tma_load_3d(dV + hf * HALF_BYTES, &tm_v, bar(BAR_VFULL + stage), hf * 64, kh, tok);
+            }
+          }
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+    }
+  } else if (warp == 9) {
+    // ======================= MMA issuer =======================
+    if (lane == 0) {
+      bool ok = mbar_wait(bar(BAR_Q), 0);
+      auto issue_S = [&](int i, int stage) {
+        tc_fence_after();
+        const uint32_t aQ = sbase + OFF_Q + i * TILE_BYTES, aK = sbase + OFF_K + stage * TILE_BYTES;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+          tc_mma_ss(tmem + i * 128, smem_desc(aQ + off, 16), smem_desc(aK + off, 16), IDESC_S, ks > 0);
+        }
+        tc_commit(bar(BAR_SFULL + i));
+      };
+      auto issue_PV = [&](int i, int stage, bool first) {
+        tc_fence_after();
+        const uint32_t aV = sbase + OFF_V + stage * TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk)
+          tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, smem_desc(aV + kk * 2048, HALF_BYTES), IDESC_PV,
+                    !(first && kk == 0));
+      };
+      if (ok) ok = mbar_wait(bar(BAR_KFULL + 0), 0);
+      if (ok) {
+        issue_S(0, 0);
+        issue_S(1, 0);
+        tc_commit(bar(BAR_KEMPTY + 0));
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int stage = j % KV_STAGES, nstage = (j + 1) % KV_STAGES;
+        const bool more = j + 1 < n_tiles;
+        ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + 0), j & 1);
+        if (!ok) break;
+        issue_PV(0, stage, j == 0);
+        if (more) {
+          ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
+          if (!ok) break;
+          issue_S(0, nstage);
+        }
+        ok = mbar_wait(bar(BAR_PFULL + 1), j & 1);
+        if (!ok) break;
+        issue_PV(1, stage, j == 0);
+        tc_commit(bar(BAR_VEMPTY + stage));
+        if (more) {
+          issue_S(1, nstage);
+          tc_commit(bar(BAR_KEMPTY + nstage));
+        }
+      }
+      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 20);
+      tc_commit(bar(BAR_OFINAL));
+    }
+  } else {
+    // ======================= softmax warps =======================
+    const int i = warp >> 2;                    // Q tile
+    const int rr = (warp & 3) * 32 + lane;      // row in the tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_addr + i * 128;
+    const uint32_t tO = tmem + lane_addr + 256 + i * 128;
+    const int ri = b * BM + rr;                 // chunk-relative row
+    const int pos = ctx + ri;                   // absolute position
+    float m_st = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + i), j & 1))) {  // warp-uniform: TMEM ops are warp-wide
+        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 30 + i);
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      // visible column interval [lo, hi) of this row in this tile; ring tiles are decided per column
+      int lo = 0, hi = BN;
+      bool ring_tile = false, masked = false;
+      if (j < seq.nA) {
+        if (!p.is_swa) {
+          hi = min(BN, ctx - j * BN);
+          masked = hi < BN;
+        } else {
+          ring_tile = true;
+          masked = true;
+        }
+      } else {
+        const int c = seq.c_lo + (j - seq.nA);
+        hi = ri - c * BN + 1;
+        hi = hi < 0 ? 0 : (hi > BN ? BN : hi);
+        if (p.is_swa) {
+          lo = ri - M.W + 1 - c * BN;
+          lo = lo < 0 ? 0 : lo;
+        }
+        masked = (c == b) || p.is_swa;
+      }
+      auto col_valid = [&](int col) -> bool {
+        if (!ring_tile) return col >= lo && col < hi;
+        const int page_in_ring = 2 * j + (col >> 6);
+        if (page_in_ring >= M.R) return false;
+        int off = page_in_ring * PG + (col & 63) - head;
+        if (off < 0) off += M.C;
+        const int kpos = ctx - M.C + off;  // position held by this slot before the chunk's append
+        return kpos >= 0 && kpos > pos - M.W;
+      };
+      // pass 1: row maximum
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t v[32];
+        tmem_ld32(tS + c4 * 32, v);
+        tc_wait_ld();
+        if (masked) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            if (col_valid(c4 * 32 + k)) mx = fmaxf(mx, __uint_as_float(v[k]));
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
+        }
+      }
+      const float mx_s = mx * M.scale_log2;
+      if (j == 0) {
+        m_st = mx_s;
+      } else {
+        const bool grow = mx_s > m_st + 8.f;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float m_new = grow ? mx_s : m_st;
+          const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_st - m_new);
+#pragma unroll 1
+          for (int c4 = 0; c4 < 4; ++c4) {
+            uint32_t v[32];
+            tmem_ld32(tO + c4 * 32, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
+            tmem_st32(tO + c4 * 32, v);
+          }
+          l_run *= alpha;
+          m_st = m_new;
+        }
+      }
+      const float m_use = (m_st == -INFINITY) ? 0.f : m_st;
+      // pass 2: probabilities -> bf16 pairs written over the first 64 columns of S
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t v[32];
+        tmem_ld32(tS + c4 * 32, v);
+        tc_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          float p0 = fast_exp2(__uint_as_float(v[2 * k]) * M.scale_log2 - m_use);
+          float p1 = fast_exp2(__uint_as_float(v[2 * k + 1]) * M.scale_log2 - m_use);
+          if (masked) {
+            p0 = col_valid(c4 * 32 + 2 * k) ? p0 : 0.f;
+            p1 = col_valid(c4 * 32 + 2 * k + 1) ? p1 : 0.f;
+          }
+          l_run += p0 + p1;
+          pk[k] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(tS + c4 * 16, pk);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(BAR_PFULL + i));
+    }
+    // ---- epilogue: O / l -> global ----
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFINAL), 0));
+    if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 40 + i);
+    tc_fence_after();
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    const bool row_ok = ok && ri < n;
+    const int64_t orow = ((int64_t)(t0 + ri) * M.Hq + (h0 + i));
+#pragma unroll 1
+    for (int c4 = 0; c4 < 4; ++c4) {
+      uint32_t v[32];
+      tmem_ld32(tO + c4 * 32, v);
+      tc_wait_ld();
+      if (row_ok) {
+        if (M.out_fp32) {
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            dst[k] = make_float4(__uint_as_float(v[4 * k]) * inv, __uint_as_float(v[4 * k + 1]) * inv,
+                                 __uint_as_float(v[4 * k + 2]) * inv, __uint_as_float(v[4 * k + 3]) * inv);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(v[8 * k]) * inv, __uint_as_float(v[8 * k + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(v[8 * k + 2]) * inv, __uint_as_float(v[8 * k + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(v[8 * k + 4]) * inv, __uint_as_float(v[8 * k + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(v[8 * k + 6]) * inv, __uint_as_float(v[8 * k + 7]) * inv);
+            dst[k] = w;
+          }
+        }
+      }
+    }
+    if (row_ok && p.lse)
+      p.lse[orow] = l_run > 0.f ? (m_st + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+  }
+
+  // ---- teardown: everyone is done with TMEM before it is released ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+}  // namespace
+
+bool hswa_prefill_tc_supported(const ModelParams& m) { return m.D == 128 && m.P == 64 && (m.G % 2) == 0; }
+
+cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                                   const CUtensorMap& tm_v, const PrefillParams& p, cudaStream_t s) {
+  if (p.b.B == 0 || p.total_q == 0 || p.max_q_len == 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int max_tiles = (p.max_q_len + BM - 1) / BM;
+  dim3 grid(p.m.G / 2, p.m.Hkv, (unsigned)(p.b.B * max_tiles));
+  prefill_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
+  return cudaGetLastError();
+}

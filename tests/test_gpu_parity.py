@@ -341,3 +341,28 @@ def test_host_side_argument_errors():
                      max_q_len=1, total_q=0)
     hb.hswa_decode_attn(h, full, empty, q, None, None, out, None, None)
     assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+
+
+# ---------------------------------------------------------------------------------------------------------
+# tcgen05 prefill kernel (head_dim 128, page 64, even GQA group)
+@pytest.mark.parametrize("case", ["one_tile", "two_tiles", "ctx_small", "ragged"])
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_prefill_tc_small(case, is_swa):
+    d = dims(2, 128, 64, 1)
+    ctx, q_len = {"one_tile": ([0], [128]), "two_tiles": ([0], [256]), "ctx_small": ([70], [128]),
+                  "ragged": ([0, 130, 64], [100, 129, 1])}[case]
+    sc = build_scenario(d, ctx, q_len, seed=31)
+    err, lerr = run_prefill(sc, is_swa)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(2, 128, 64, 3), dims(4, 128, 64, 1)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_prefill_tc_sweep(d, is_swa):
+    ctx = [0, 1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 500, 5000]
+    q_len = [300, 128, 129, 1, 127, 256, 64, 700, 0, 5, 130, 257, 400]
+    sc = build_scenario(d, ctx, q_len, seed=32)
+    err, lerr = run_prefill(sc, is_swa)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+    err, _ = run_prefill(sc, is_swa, fuse_append=False, out_dtype=torch.bfloat16)
+    assert err <= 2 * TOL, err   # bf16 output: rows with 1-3 keys can carry half a bf16 ulp of a value near 4
