@@ -37,6 +37,7 @@ def parse_args():
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
+    ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill block reported under 'extra'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -60,12 +61,14 @@ def stored_traffic(key):
     return None
 
 
-def make_workload(name, seed_offset=0, layers=0, batch=0):
+def make_workload(name, seed_offset=0, layers=0, batch=0, chunk=0):
     from paper_2607_13095_b200 import workloads as wl
     kw = {"batch": batch} if batch else {}
     if name == "cfg2":
         return wl.config2(seed=2 + seed_offset, **kw)
     if name == "cfg3":
+        if chunk:
+            kw["chunk"] = chunk
         return wl.config3(seed=3 + seed_offset, **kw)
     if name == "cfg4":
         return wl.config4(seed=4 + seed_offset, **kw)
@@ -340,6 +343,78 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks):
+    """--workload cfg3: the chunked-prefill block as the measured workload (value = attention TFLOP/s of the
+    whole 1 Full + 6 SWA block, fused append included)."""
+    from paper_2607_13095_b200 import accounting
+    from paper_2607_13095_b200 import binding as hb
+    w = make_workload("cfg3", seed_offset=rank, batch=args.batch, chunk=args.chunk)
+    pb = PrefillBench(w, device)
+    t, d = w.tables, w.dims
+    full_i = w.layer_is_swa.index(False)
+    L = len(w.layer_is_swa)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(events=None):
+        for i in range(L):
+            timed = events is not None and i == full_i
+            if timed:
+                events[0].record()
+            pb.run_layer(i)
+            if timed:
+                events[1].record()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        e0.record()
+        for k in range(args.steps):
+            step(ev[k])
+        e1.record()
+        torch.cuda.synchronize()
+    barrier()
+    st = hb.hswa_get_async_error(pb.h)
+    if st[0] != hb.HSWA_OK:
+        raise SystemExit(f"device error word set during the timed region: {st}")
+    tmax = torch.tensor([e0.elapsed_time(e1)], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    ms_step = float(tmax.item()) / args.steps
+    full_ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    f_full, f_swa = accounting.prefill_flops(w, False), accounting.prefill_flops(w, True)
+    n_full = sum(1 for s in w.layer_is_swa if not s)
+    flops_step = n_full * f_full + (L - n_full) * f_swa
+    if rank != 0:
+        return
+    achieved = f_full / (full_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    line = {
+        "metric": "prefill_attn_tflops", "value": flops_step * world / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "swa_layers": int(sum(w.layer_is_swa)), "batch": t.batch,
+                   "chunk": int(t.q_len.max()), "ctx": [int(x) for x in t.ctx_len], "num_q_heads": d.num_q_heads,
+                   "num_kv_heads": d.num_kv_heads, "head_dim": d.head_dim, "page_size": d.page_size,
+                   "l2": "inputs larger than L2 (Q, K/V chunk and output tensors are 1.07 GB + 0.27 GB + 1.07 GB)"},
+        "tokens_per_s": t.total_q * world / (ms_step * 1e-3),
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": stored_traffic("prefill_full_cfg3"), "kernel": "prefill_tc_kernel (+ append_kernel), one Full layer",
+                     "ms_per_launch": full_ms, "algorithmic_flops_per_launch": f_full, "peak_source": peaks["source"]
+                     + " (sustained cuBLAS bf16; kernel timed inside a long step)",
+                     "frac_of_measured_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0},
+        "clocks": clocks.summary(), "e2e": None, "gpu_launches": 2 * L * args.steps,
+    }
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -363,7 +438,8 @@ def main():
     peaks = measured_peaks()
 
     if args.workload == "cfg3":
-        raise SystemExit("cfg3 is reported under 'extra' of the default run; use --workload cfg2|cfg4|cfg5")
+        run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks)
+        return
     w = make_workload(args.workload, seed_offset=rank, layers=args.layers, batch=args.batch)
     total_steps = args.steps + args.warmup
     bench = DecodeBench(w, 2 * total_steps + 8, device)

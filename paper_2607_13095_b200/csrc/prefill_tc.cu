@@ -86,7 +86,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
   return d;
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -98,7 +104,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
       : "r"(addr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -356,22 +362,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         const int kpos = ctx - M.C + off;  // position held by this slot before the chunk's append
         return kpos >= 0 && kpos > pos - M.W;
       };
-      // pass 1: row maximum
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
-        uint32_t v[32];
-        tmem_ld32(tS + c4 * 32, v);
-        tc_wait_ld();
-        if (masked) {
+      // the whole row of scores: one round trip to TMEM
+      uint32_t v[128];
+      tmem_ld32(tS, v);
+      tmem_ld32(tS + 32, v + 32);
+      tmem_ld32(tS + 64, v + 64);
+      tmem_ld32(tS + 96, v + 96);
+      tc_wait_ld();
+      if (masked) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k)
-            if (col_valid(c4 * 32 + k)) mx = fmaxf(mx, __uint_as_float(v[k]));
-        } else {
-#pragma unroll
-          for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
-        }
+        for (int k = 0; k < 128; ++k)
+          if (!col_valid(k)) v[k] = 0xff800000u;  // -inf
       }
+      float mx = fmaxf(__uint_as_float(v[0]), __uint_as_float(v[1]));
+#pragma unroll
+      for (int k = 2; k < 128; k += 2) mx = max3(mx, __uint_as_float(v[k]), __uint_as_float(v[k + 1]));
       const float mx_s = mx * M.scale_log2;
       if (j == 0) {
         m_st = mx_s;
@@ -382,38 +387,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
           const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_st - m_new);
 #pragma unroll 1
           for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t v[32];
-            tmem_ld32(tO + c4 * 32, v);
+            uint32_t w[32];
+            tmem_ld32(tO + c4 * 32, w);
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
-            tmem_st32(tO + c4 * 32, v);
+            for (int k = 0; k < 32; ++k) w[k] = __float_as_uint(__uint_as_float(w[k]) * alpha);
+            tmem_st32(tO + c4 * 32, w);
           }
           l_run *= alpha;
           m_st = m_new;
         }
       }
       const float m_use = (m_st == -INFINITY) ? 0.f : m_st;
-      // pass 2: probabilities -> bf16 pairs written over the first 64 columns of S
-#pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
-        uint32_t v[32];
-        tmem_ld32(tS + c4 * 32, v);
-        tc_wait_ld();
-        uint32_t pk[16];
+      // probabilities -> bf16 pairs written over the first 64 columns of S (packed two-wide fp32 math)
+      const float2 sc2 = make_float2(M.scale_log2, M.scale_log2), nm2 = make_float2(-m_use, -m_use);
+      float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          float p0 = fast_exp2(__uint_as_float(v[2 * k]) * M.scale_log2 - m_use);
-          float p1 = fast_exp2(__uint_as_float(v[2 * k + 1]) * M.scale_log2 - m_use);
-          if (masked) {
-            p0 = col_valid(c4 * 32 + 2 * k) ? p0 : 0.f;
-            p1 = col_valid(c4 * 32 + 2 * k + 1) ? p1 : 0.f;
-          }
-          l_run += p0 + p1;
-          pk[k] = pack_bf16x2(p0, p1);
-        }
-        tmem_st16(tS + c4 * 16, pk);
+      for (int k = 0; k < 64; ++k) {
+        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
+        const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+        acc = __fadd2_rn(acc, e);
+        v[k] = pack_bf16x2(e.x, e.y);
       }
+      l_run += acc.x + acc.y;
+      tmem_st32(tS, v);
+      tmem_st32(tS + 32, v + 32);
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_PFULL + i));
