@@ -89,11 +89,12 @@ hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtenso
 }
 
 // 3-D view of a [T][heads][D] activation tensor for TMA: box {64, 1, box_rows}, 128-byte swizzle.
-hswa_status make_rows_map(const hswa_handle* h, const void* ptr, int heads, int64_t rows, int box_rows, CUtensorMap* tm) {
+hswa_status make_rows_map(const hswa_handle* h, const void* ptr, int heads, int64_t rows, int box_rows, CUtensorMap* tm,
+                          int box_heads = 1) {
   const cuuint64_t D = (cuuint64_t)h->cfg.head_dim;
   cuuint64_t dims[3] = {D, (cuuint64_t)heads, (cuuint64_t)rows};
   cuuint64_t strides[2] = {D * 2, D * 2 * (cuuint64_t)heads};
-  cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult rc = h->encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -300,7 +301,22 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
     if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->total_q, 128, &tm_q)) != HSWA_OK) return st;
     if ((st = make_rows_map(h, k_new, h->cfg.num_kv_heads, b->total_q, 128, &tm_k)) != HSWA_OK) return st;
     if ((st = make_rows_map(h, v_new, h->cfg.num_kv_heads, b->total_q, 128, &tm_v)) != HSWA_OK) return st;
-    if (hswa_launch_prefill_tc(tm_pool, tm_q, tm_k, tm_v, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+    // SWA layers: tokens whose whole window lies inside the chunk go to the GQA-packed kernel; the first
+    // tokens (which also read the ring) stay on the general tile kernel.
+    int tq = 0, nkeys = 0;
+    hswa_prefill_packed_geometry(h->group, &tq, &nkeys);
+    const int split_tiles = (h->cfg.window - 1 + 127) / 128;  // 128-token tiles that can reach below the chunk
+    const bool packed = layer->is_swa && tq > 0 && h->cfg.window <= 128 && b->max_q_len > split_tiles * 128;
+    if (hswa_launch_prefill_tc(tm_pool, tm_q, tm_k, tm_v, p, packed ? split_tiles : 0, (cudaStream_t)stream) != cudaSuccess)
+      return HSWA_ERR_CUDA;
+    if (packed) {
+      CUtensorMap pq, pk, pv;
+      if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->total_q, tq, &pq, h->group)) != HSWA_OK) return st;
+      if ((st = make_rows_map(h, k_new, h->cfg.num_kv_heads, b->total_q, nkeys, &pk)) != HSWA_OK) return st;
+      if ((st = make_rows_map(h, v_new, h->cfg.num_kv_heads, b->total_q, nkeys, &pv)) != HSWA_OK) return st;
+      if (hswa_launch_prefill_swa_packed(pq, pk, pv, p, split_tiles * 128, (cudaStream_t)stream) != cudaSuccess)
+        return HSWA_ERR_CUDA;
+    }
   } else {
     if (hswa_launch_prefill_mma(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   }

@@ -94,7 +94,10 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
 bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                                   const CUtensorMap& tm_v, const PrefillParams& p, cudaStream_t s);
+                                   const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s);
+void hswa_prefill_packed_geometry(int G, int* tq, int* nkeys);
+cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                           const PrefillParams& p, int first_tok, cudaStream_t s);
 cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,
                                 const int32_t* q_indptr, cudaStream_t s);
 cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,

@@ -147,7 +147,7 @@ __device__ __forceinline__ TileSeq tile_seq(int is_swa, int ctx, int b, int W, i
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_constant__ CUtensorMap tm_q,
                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                  const PrefillParams p, const int max_tiles) {
+                  const PrefillParams p, const int max_tiles) {  // tiles b < max_tiles only
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[NUM_BARS];
   __shared__ uint32_t tmem_base_slot;
@@ -462,16 +462,245 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   }
 }
 
+
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(addr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(addr)
+               : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// SWA layers, tokens whose whole window lies inside the chunk (paper Sec. 2.1: an SWA layer attends to W keys
+// only, so the work per token is constant and the layer is bound by moving Q and the output, not by the
+// tensor cores).  GQA-packed: one block = TQ = 128 / G consecutive tokens x the G query heads of one KV head
+// (128 rows), against the TQ + W - 1 keys those tokens can see, rounded up to N.  One S MMA group, one
+// softmax, one PV MMA group; K and V are loaded once for all G heads.  TMEM: S in columns [0, N), P over its
+// first N / 2 columns, O in columns [128, 256) (it overlaps the tail of S, which is dead by then), 256 columns
+// per block so that two blocks share an SM and hide each other's load and hand-off latencies.
+template <int G>
+struct PackedCfg {
+  static constexpr int TQ = 128 / G;                          // tokens per block
+  static constexpr int N = ((TQ + 128 - 1 + 15) / 16) * 16;   // keys per block for W <= 128
+  static constexpr int KV_HALF = N * 128;                     // bytes of one 64-element half of the K or V tile
+  static constexpr int KV_BYTES = 2 * KV_HALF;
+  static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = OFF_K + KV_BYTES;
+  static constexpr int SMEM = OFF_V + KV_BYTES + 1024;
+  static constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+};
+
+template <int G>
+__global__ void __launch_bounds__(192, 2)
+prefill_swa_packed_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                          const __grid_constant__ CUtensorMap tm_v, const PrefillParams p, const int first_tok) {
+  using C = PackedCfg<G>;
+  constexpr int TQ = C::TQ, N = C::N;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[6];
+  __shared__ uint32_t tmem_base_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const ModelParams& M = p.m;
+  enum { B_Q = 0, B_K = 1, B_V = 2, B_S = 3, B_P = 4, B_O = 5 };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kh = blockIdx.x, r = blockIdx.z;
+  const int t0 = p.b.q_indptr[r];
+  const int n = p.b.q_indptr[r + 1] - t0;
+  const int i0 = first_tok + (int)blockIdx.y * TQ;  // first chunk-relative token of this block
+  if (i0 >= n) return;
+  if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;
+  const int key0 = i0 - (M.W - 1);  // chunk-relative index of key column 0 (>= 0 by construction)
+
+  auto bar = [&](int i) { return smem_u32(&bars[i]); };
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_Q), 1);
+    mbar_init(bar(B_K), 1);
+    mbar_init(bar(B_V), 1);
+    mbar_init(bar(B_S), 1);
+    mbar_init(bar(B_P), 128);
+    mbar_init(bar(B_O), 1);
+    mbar_fence_init();
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(256)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar(B_Q), TILE_BYTES);
+      mbar_arrive_expect_tx(bar(B_K), C::KV_BYTES);
+      mbar_arrive_expect_tx(bar(B_V), C::KV_BYTES);
+      for (int hf = 0; hf < 2; ++hf) {
+        tma_load_3d(sbase + C::OFF_Q + hf * HALF_BYTES, &tm_q, bar(B_Q), hf * 64, kh * G, t0 + i0);
+        tma_load_3d(sbase + C::OFF_K + hf * C::KV_HALF, &tm_k, bar(B_K), hf * 64, kh, t0 + key0);
+      }
+      for (int hf = 0; hf < 2; ++hf) tma_load_3d(sbase + C::OFF_V + hf * C::KV_HALF, &tm_v, bar(B_V), hf * 64, kh, t0 + key0);
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      bool ok = mbar_wait(bar(B_Q), 0) && mbar_wait(bar(B_K), 0);
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t qoff = (ks >> 2) * HALF_BYTES + (ks & 3) * 32, koff = (ks >> 2) * C::KV_HALF + (ks & 3) * 32;
+          tc_mma_ss(tmem, smem_desc(sbase + C::OFF_Q + qoff, 16), smem_desc(sbase + C::OFF_K + koff, 16), C::IDESC_S, ks > 0);
+        }
+        tc_commit(bar(B_S));
+        ok = mbar_wait(bar(B_V), 0) && mbar_wait(bar(B_P), 0);
+      }
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < N / 16; ++kk)
+          tc_mma_ts(tmem + 128, tmem + kk * 8, smem_desc(sbase + C::OFF_V + kk * 2048, C::KV_HALF), IDESC_PV, kk > 0);
+      } else {
+        record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 50);
+      }
+      tc_commit(bar(B_O));
+    }
+  } else {
+    const int rr = warp * 32 + lane;             // row = TMEM lane
+    const int tl = rr / G, g = rr % G;           // local token, head in group
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const uint32_t tS = tmem + lane_addr, tO = tmem + lane_addr + 128;
+    const int lo = tl, hi = tl + M.W;            // visible key columns [lo, hi)
+    bool ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S), 0));
+    float mx = -INFINITY, l_run = 0.f, m_use = 0.f;
+    if (ok) {
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < N / 16; ++c) {
+        uint32_t v[16];
+        tmem_ld16(tS + c * 16, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int col = c * 16 + k;
+          if (col >= lo && col < hi) mx = fmaxf(mx, __uint_as_float(v[k]));
+        }
+      }
+      m_use = mx == -INFINITY ? 0.f : mx * M.scale_log2;
+#pragma unroll 1
+      for (int c = 0; c < N / 16; ++c) {
+        uint32_t v[16];
+        tmem_ld16(tS + c * 16, v);
+        tc_wait_ld();
+        uint32_t pk[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int col = c * 16 + 2 * k;
+          float p0 = fast_exp2(__uint_as_float(v[2 * k]) * M.scale_log2 - m_use);
+          float p1 = fast_exp2(__uint_as_float(v[2 * k + 1]) * M.scale_log2 - m_use);
+          p0 = (col >= lo && col < hi) ? p0 : 0.f;
+          p1 = (col + 1 >= lo && col + 1 < hi) ? p1 : 0.f;
+          l_run += p0 + p1;
+          pk[k] = pack_bf16x2(p0, p1);
+        }
+        tmem_st8(tS + c * 8, pk);
+      }
+      tc_wait_st();
+    } else if (lane == 0) {
+      record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 51);
+    }
+    tc_fence_before();
+    mbar_arrive(bar(B_P));
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_O), 0));
+    tc_fence_after();
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    const bool row_ok = ok && (i0 + tl) < n;
+    const int64_t orow = (int64_t)(t0 + i0 + tl) * M.Hq + kh * G + g;
+#pragma unroll 1
+    for (int c4 = 0; c4 < 4; ++c4) {
+      uint32_t v[32];
+      tmem_ld32(tO + c4 * 32, v);
+      tc_wait_ld();
+      if (row_ok) {
+        if (M.out_fp32) {
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            dst[k] = make_float4(__uint_as_float(v[4 * k]) * inv, __uint_as_float(v[4 * k + 1]) * inv,
+                                 __uint_as_float(v[4 * k + 2]) * inv, __uint_as_float(v[4 * k + 3]) * inv);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(v[8 * k]) * inv, __uint_as_float(v[8 * k + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(v[8 * k + 2]) * inv, __uint_as_float(v[8 * k + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(v[8 * k + 4]) * inv, __uint_as_float(v[8 * k + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(v[8 * k + 6]) * inv, __uint_as_float(v[8 * k + 7]) * inv);
+            dst[k] = w;
+          }
+        }
+      }
+    }
+    if (row_ok && p.lse) p.lse[orow] = l_run > 0.f ? (m_use + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+  }
+}
+
+template <int G>
+cudaError_t launch_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const PrefillParams& p,
+                          int first_tok, cudaStream_t s) {
+  using C = PackedCfg<G>;
+  auto kern = prefill_swa_packed_kernel<G>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+  if (e != cudaSuccess) return e;
+  const int tiles = (p.max_q_len - first_tok + C::TQ - 1) / C::TQ;
+  dim3 grid(p.m.Hkv, tiles, p.b.B);
+  kern<<<grid, 192, C::SMEM, s>>>(tm_q, tm_k, tm_v, p, first_tok);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool hswa_prefill_tc_supported(const ModelParams& m) { return m.D == 128 && m.P == 64 && (m.G % 2) == 0; }
 
+// Geometry of the GQA-packed SWA kernel for group size G: tokens per block and keys per block (0 = unsupported).
+void hswa_prefill_packed_geometry(int G, int* tq, int* nkeys) {
+  *tq = 0;
+  *nkeys = 0;
+  if (G == 8) { *tq = PackedCfg<8>::TQ; *nkeys = PackedCfg<8>::N; }
+  if (G == 4) { *tq = PackedCfg<4>::TQ; *nkeys = PackedCfg<4>::N; }
+}
+
+cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                           const PrefillParams& p, int first_tok, cudaStream_t s) {
+  if (p.b.B == 0 || p.max_q_len <= first_tok) return cudaSuccess;
+  if (p.m.G == 8) return launch_packed<8>(tm_q, tm_k, tm_v, p, first_tok, s);
+  if (p.m.G == 4) return launch_packed<4>(tm_q, tm_k, tm_v, p, first_tok, s);
+  return cudaErrorInvalidValue;
+}
+
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                                   const CUtensorMap& tm_v, const PrefillParams& p, cudaStream_t s) {
+                                   const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s) {
   if (p.b.B == 0 || p.total_q == 0 || p.max_q_len == 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  const int max_tiles = (p.max_q_len + BM - 1) / BM;
+  int max_tiles = (p.max_q_len + BM - 1) / BM;
+  if (tile_limit > 0 && tile_limit < max_tiles) max_tiles = tile_limit;
   dim3 grid(p.m.G / 2, p.m.Hkv, (unsigned)(p.b.B * max_tiles));
   prefill_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
   return cudaGetLastError();
