@@ -5,10 +5,11 @@
 //
 // One thread block = 128 query tokens x 2 query heads of one GQA group (two 128-row Q tiles that share every
 // K/V tile and every mask).  Warp roles:
-//   warps 0-3   softmax for Q tile 0 (one thread per row: TMEM lane = row, so row max / row sum are thread-local)
-//   warps 4-7   softmax for Q tile 1
-//   warp  8     TMA producer: Q once, then 128-key K and V tiles through two 2-stage rings
-//   warp  9     MMA issuer: S_i = Q_i K^T (SS form), O_i += P_i V (TS form, P read from TMEM where it
+//   warps 0-7   softmax for Q tile 0: TMEM lane = row; two warps share each 32-row lane quadrant and take 64 key
+//               columns each, exchanging partial row maxima / sums through shared memory
+//   warps 8-15  softmax for Q tile 1
+//   warp  16    TMA producer: Q once, then 128-key K and V tiles through two 2-stage rings
+//   warp  17    MMA issuer: S_i = Q_i K^T (SS form), O_i += P_i V (TS form, P read from TMEM where it
 //               overwrites S_i), in the order PV0(j), S0(j+1), PV1(j), S1(j+1) so that one tile's softmax
 //               overlaps the other tile's MMAs
 // TMEM columns: S0 0-127, S1 128-255, O0 256-383, O1 384-511 (all fp32; P_i = bf16 pairs in the first 64
@@ -30,7 +31,7 @@ constexpr int PG = 64;                // page size
 constexpr int HALF_BYTES = 128 * 128; // [128 rows][128 B]: one 64-element half of a 128-row tile
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int KV_STAGES = 2;
-constexpr int NUM_THREADS = 320;
+constexpr int NUM_THREADS = 576;  // 16 softmax warps + producer + MMA issuer
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                  // 2 Q tiles
@@ -41,6 +42,19 @@ constexpr int SMEM_BYTES = SMEM_TILES + 1024;
 
 constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [key][d] with d contiguous
+
+// Of every HSWA_POLY_DEN element pairs, HSWA_POLY_NUM take 2^x on the FMA pipe instead of the MUFU.
+#ifndef HSWA_POLY_NUM
+#define HSWA_POLY_NUM 1
+#define HSWA_POLY_DEN 2
+#endif
+
+#ifdef HSWA_PROBE_TRACE
+__device__ long long hswa_trace[16 * 64];
+#define TRACE(slot, j) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (j) < 64) hswa_trace[(slot) * 64 + (j)] = clock64(); } while (0)
+#else
+#define TRACE(slot, j) do { } while (0)
+#endif
 
 // barrier indices
 enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PFULL = 11,
@@ -124,6 +138,18 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t addr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(addr)
+               : "memory");
+}
+
 // The sequence of key tiles one block walks: nA cached tiles, then chunk tiles c_lo .. c_lo + nB - 1.
 struct TileSeq {
   int nA, c_lo, nB;
@@ -151,6 +177,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[NUM_BARS];
   __shared__ uint32_t tmem_base_slot;
+  __shared__ float xch[2][2][2][128];  // [parity][Q tile][column half][row]: partial row maxima / sums
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
@@ -181,12 +208,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_PFULL + i), 128);
+      mbar_init(bar(BAR_PFULL + i), 8);  // one arrival per softmax warp
     }
     mbar_init(bar(BAR_OFINAL), 1);
     mbar_fence_init();
   }
-  if (warp == 8) {
+  if (warp == 16) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -196,7 +223,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
-  if (warp == 8) {
+  if (warp == 16) {
     // ======================= TMA producer =======================
     if (lane == 0) {
       tma_prefetch_desc(&tm_pool);
@@ -263,7 +290,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     // ======================= MMA issuer =======================
     if (lane == 0) {
       bool ok = mbar_wait(bar(BAR_Q), 0);
@@ -296,42 +323,54 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         const bool more = j + 1 < n_tiles;
         ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + 0), j & 1);
         if (!ok) break;
+        TRACE(0, j);
         issue_PV(0, stage, j == 0);
         if (more) {
           ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
           if (!ok) break;
           issue_S(0, nstage);
         }
+        TRACE(1, j);
         ok = mbar_wait(bar(BAR_PFULL + 1), j & 1);
         if (!ok) break;
+        TRACE(2, j);
         issue_PV(1, stage, j == 0);
         tc_commit(bar(BAR_VEMPTY + stage));
         if (more) {
           issue_S(1, nstage);
           tc_commit(bar(BAR_KEMPTY + nstage));
         }
+        TRACE(3, j);
       }
       if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 20);
       tc_commit(bar(BAR_OFINAL));
     }
   } else {
     // ======================= softmax warps =======================
-    const int i = warp >> 2;                    // Q tile
-    const int rr = (warp & 3) * 32 + lane;      // row in the tile = TMEM lane
-    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_addr + i * 128;
-    const uint32_t tO = tmem + lane_addr + 256 + i * 128;
+    // 8 warps per Q tile: warp pair (quad, half) shares the 32 rows of a TMEM lane quadrant and splits the 128
+    // key columns in two, so four softmax warps are resident per scheduler and hide each other's MUFU and
+    // TMEM latencies.  The halves of a row exchange their partial maxima through shared memory.
+    const int i = warp >> 3;                    // Q tile
+    const int quad = warp & 3, half = (warp >> 2) & 1;
+    const int rr = quad * 32 + lane;            // row in the tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tS = tmem + lane_addr + i * 128 + half * 64;
+    const uint32_t tP = tmem + lane_addr + i * 128 + half * 32;
+    const uint32_t tO = tmem + lane_addr + 256 + i * 128 + half * 64;
+    const int pair_bar = 1 + i * 4 + quad;      // named barrier of the two warps that share these rows
     const int ri = b * BM + rr;                 // chunk-relative row
     const int pos = ctx + ri;                   // absolute position
     float m_st = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
-      if (!__all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + i), j & 1))) {  // warp-uniform: TMEM ops are warp-wide
-        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 30 + i);
-        ok = false;
-        break;
-      }
-      tc_fence_after();
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + i), j & 1));  // warp-uniform: TMEM ops are warp-wide
+      if (lane == 0 && (warp & 7) == 0) TRACE(4 + 6 * i, j);
+#ifdef HSWA_PROBE_NO_SOFTMAX
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));
+      continue;
+#endif
       // visible column interval [lo, hi) of this row in this tile; ring tiles are decided per column
       int lo = 0, hi = BN;
       bool ring_tile = false, masked = false;
@@ -353,30 +392,71 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         }
         masked = (c == b) || p.is_swa;
       }
-      auto col_valid = [&](int col) -> bool {
-        if (!ring_tile) return col >= lo && col < hi;
-        const int page_in_ring = 2 * j + (col >> 6);
-        if (page_in_ring >= M.R) return false;
-        int off = page_in_ring * PG + (col & 63) - head;
-        if (off < 0) off += M.C;
-        const int kpos = ctx - M.C + off;  // position held by this slot before the chunk's append
-        return kpos >= 0 && kpos > pos - M.W;
-      };
-      // the whole row of scores: one round trip to TMEM
-      uint32_t v[128];
-      tmem_ld32(tS, v);
-      tmem_ld32(tS + 32, v + 32);
-      tmem_ld32(tS + 64, v + 64);
-      tmem_ld32(tS + 96, v + 96);
-      tc_wait_ld();
+      // bit k of (vm_lo, vm_hi) = this thread's column half * 64 + k is visible to this row
+      uint32_t vm_lo = 0xffffffffu, vm_hi = 0xffffffffu;
       if (masked) {
-#pragma unroll
-        for (int k = 0; k < 128; ++k)
-          if (!col_valid(k)) v[k] = 0xff800000u;  // -inf
+        if (!ring_tile) {
+          int c0 = lo - half * 64, c1 = hi - half * 64;
+          c0 = c0 < 0 ? 0 : (c0 > 64 ? 64 : c0);
+          c1 = c1 < 0 ? 0 : (c1 > 64 ? 64 : c1);
+          const uint64_t below_c1 = c1 >= 64 ? ~0ull : ((1ull << c1) - 1);
+          const uint64_t below_c0 = c0 >= 64 ? ~0ull : ((1ull << c0) - 1);
+          const uint64_t vm = c1 > c0 ? (below_c1 & ~below_c0) : 0ull;
+          vm_lo = (uint32_t)vm;
+          vm_hi = (uint32_t)(vm >> 32);
+        } else {
+          // ring tile: ring page 2j + half; slot -> position it held before the chunk's append
+          uint64_t vm = 0;
+          const int page_in_ring = 2 * j + half;
+          if (page_in_ring < M.R) {
+#pragma unroll 1
+            for (int k = 0; k < 64; ++k) {
+              int off = page_in_ring * PG + k - head;
+              if (off < 0) off += M.C;
+              const int kpos = ctx - M.C + off;
+              if (kpos >= 0 && kpos > pos - M.W) vm |= 1ull << k;
+            }
+          }
+          vm_lo = (uint32_t)vm;
+          vm_hi = (uint32_t)(vm >> 32);
+        }
       }
-      float mx = fmaxf(__uint_as_float(v[0]), __uint_as_float(v[1]));
+      // this thread's 64 scores: one round trip to TMEM
+      uint32_t v[64];
+      float mx = INFINITY;  // +inf tells the partner warp that this warp gave up
+      if (ok) {
+        tc_fence_after();
+        tmem_ld32(tS, v);
+        tmem_ld32(tS + 32, v + 32);
+        tc_wait_ld();
+        if (masked) {
 #pragma unroll
-      for (int k = 2; k < 128; k += 2) mx = max3(mx, __uint_as_float(v[k]), __uint_as_float(v[k + 1]));
+          for (int k = 0; k < 32; ++k) {
+            if (!((vm_lo >> k) & 1u)) v[k] = 0xff800000u;  // -inf
+            if (!((vm_hi >> k) & 1u)) v[32 + k] = 0xff800000u;
+          }
+        }
+        float mx4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mx4[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+#pragma unroll
+        for (int k = 8; k < 64; k += 8) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mx4[c] = max3(mx4[c], __uint_as_float(v[k + 2 * c]), __uint_as_float(v[k + 2 * c + 1]));
+        }
+        mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      }
+      if (lane == 0 && (warp & 7) == 0) TRACE(5 + 6 * i, j);
+      xch[j & 1][i][half][rr] = mx;
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+      const float other = xch[j & 1][i][half ^ 1][rr];
+      if (!ok || __any_sync(0xffffffffu, other == INFINITY)) {
+        if (lane == 0 && !ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 30 + i);
+        ok = false;
+        break;
+      }
+      if (lane == 0 && (warp & 7) == 0) TRACE(6 + 6 * i, j);
+      mx = fmaxf(mx, other);
       const float mx_s = mx * M.scale_log2;
       if (j == 0) {
         m_st = mx_s;
@@ -386,13 +466,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
           const float m_new = grow ? mx_s : m_st;
           const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_st - m_new);
 #pragma unroll 1
-          for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t w[32];
-            tmem_ld32(tO + c4 * 32, w);
+          for (int c8 = 0; c8 < 8; ++c8) {  // small chunks: the 64 scores stay live in registers meanwhile
+            uint32_t w[8];
+            tmem_ld8(tO + c8 * 8, w);
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) w[k] = __float_as_uint(__uint_as_float(w[k]) * alpha);
-            tmem_st32(tO + c4 * 32, w);
+            for (int k = 0; k < 8; ++k) w[k] = __float_as_uint(__uint_as_float(w[k]) * alpha);
+            tmem_st8(tO + c8 * 8, w);
           }
           l_run *= alpha;
           m_st = m_new;
@@ -401,62 +481,90 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       const float m_use = (m_st == -INFINITY) ? 0.f : m_st;
       // probabilities -> bf16 pairs written over the first 64 columns of S (packed two-wide fp32 math)
       const float2 sc2 = make_float2(M.scale_log2, M.scale_log2), nm2 = make_float2(-m_use, -m_use);
-      float2 acc = make_float2(0.f, 0.f);
+      float2 acc[4];
 #pragma unroll
-      for (int k = 0; k < 64; ++k) {
+      for (int c = 0; c < 4; ++c) acc[c] = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < 32; ++k) {
         const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
-        const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
-        acc = __fadd2_rn(acc, e);
+        float2 e;
+        if ((k % HSWA_POLY_DEN) < HSWA_POLY_NUM) {
+          // 2^x on the FMA pipe: x = n + f with |f| <= 1/2 (magic-number rounding), cubic for 2^f (relative
+          // error 7.5e-5, far below bf16 rounding), n added into the exponent field.  The 16-lane MUFU would
+          // otherwise need 1024 clocks per 128 x 128 tile, about as long as the tile's four MMAs.
+          const float2 xc = make_float2(fmaxf(x.x, -126.f), fmaxf(x.y, -126.f));
+          const float2 t = __fadd2_rn(xc, make_float2(12582912.f, 12582912.f));
+          const float2 nf = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+          const float2 f = __fadd2_rn(xc, make_float2(-nf.x, -nf.y));
+          float2 pl = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.242611125f, 0.242611125f));
+          pl = __ffma2_rn(pl, f, make_float2(0.693260968f, 0.693260968f));
+          pl = __ffma2_rn(pl, f, make_float2(0.999928057f, 0.999928057f));
+          e.x = __uint_as_float(__float_as_uint(pl.x) + (__float_as_uint(t.x) << 23));
+          e.y = __uint_as_float(__float_as_uint(pl.y) + (__float_as_uint(t.y) << 23));
+        } else {
+          e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+        }
+        acc[k & 3] = __fadd2_rn(acc[k & 3], e);
         v[k] = pack_bf16x2(e.x, e.y);
       }
-      l_run += acc.x + acc.y;
-      tmem_st32(tS, v);
-      tmem_st32(tS + 32, v + 32);
+      const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+      l_run += (a01.x + a01.y) + (a23.x + a23.y);
+      if (lane == 0 && (warp & 7) == 0) TRACE(7 + 6 * i, j);
+      tmem_st32(tP, v);
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar(BAR_PFULL + i));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));  // 32 arrivals on one barrier word would serialise
+      if (lane == 0 && (warp & 7) == 0) TRACE(8 + 6 * i, j);
     }
     // ---- epilogue: O / l -> global ----
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFINAL), 0));
     if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 40 + i);
     tc_fence_after();
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    // the two halves of a row add up their partial sums (a warp that gave up posts NaN so both halves skip)
+    xch[0][i][half][rr] = ok ? l_run : NAN;
+    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+    const float l_other = xch[0][i][half ^ 1][rr];
+    ok = ok && !__any_sync(0xffffffffu, l_other != l_other);
+    const float l_tot = l_run + l_other;
+    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
     const bool row_ok = ok && ri < n;
     const int64_t orow = ((int64_t)(t0 + ri) * M.Hq + (h0 + i));
 #pragma unroll 1
-    for (int c4 = 0; c4 < 4; ++c4) {
-      uint32_t v[32];
-      tmem_ld32(tO + c4 * 32, v);
+    for (int c2 = 0; c2 < 2; ++c2) {
+      uint32_t w[32];
+      tmem_ld32(tO + c2 * 32, w);
       tc_wait_ld();
       if (row_ok) {
+        const int col0 = half * 64 + c2 * 32;
         if (M.out_fp32) {
-          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + c4 * 32);
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + col0);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            dst[k] = make_float4(__uint_as_float(v[4 * k]) * inv, __uint_as_float(v[4 * k + 1]) * inv,
-                                 __uint_as_float(v[4 * k + 2]) * inv, __uint_as_float(v[4 * k + 3]) * inv);
+            dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
+                                 __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
         } else {
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + c4 * 32);
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + col0);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(v[8 * k]) * inv, __uint_as_float(v[8 * k + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(v[8 * k + 2]) * inv, __uint_as_float(v[8 * k + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(v[8 * k + 4]) * inv, __uint_as_float(v[8 * k + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(v[8 * k + 6]) * inv, __uint_as_float(v[8 * k + 7]) * inv);
-            dst[k] = w;
+            uint4 u;
+            u.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
+            u.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
+            u.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
+            u.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
+            dst[k] = u;
           }
         }
       }
     }
-    if (row_ok && p.lse)
-      p.lse[orow] = l_run > 0.f ? (m_st + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+    if (row_ok && half == 0 && p.lse)
+      p.lse[orow] = l_tot > 0.f ? (m_st + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
   }
 
   // ---- teardown: everyone is done with TMEM before it is released ----
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 16) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
   }
@@ -471,11 +579,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t* r) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(addr)
       : "memory");
-}
-__device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t* r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
-               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(addr)
-               : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -526,7 +629,7 @@ prefill_swa_packed_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     mbar_init(bar(B_K), 1);
     mbar_init(bar(B_V), 1);
     mbar_init(bar(B_S), 1);
-    mbar_init(bar(B_P), 128);
+    mbar_init(bar(B_P), 4);
     mbar_init(bar(B_O), 1);
     mbar_fence_init();
   }
@@ -619,7 +722,8 @@ prefill_swa_packed_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
       record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 51);
     }
     tc_fence_before();
-    mbar_arrive(bar(B_P));
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(B_P));
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_O), 0));
     tc_fence_after();
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
@@ -675,6 +779,12 @@ cudaError_t launch_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, cons
 }
 
 }  // namespace
+
+#ifdef HSWA_PROBE_TRACE
+extern "C" int hswa_debug_read_trace(long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, hswa_trace, sizeof(long long) * 16 * 64);
+}
+#endif
 
 bool hswa_prefill_tc_supported(const ModelParams& m) { return m.D == 128 && m.P == 64 && (m.G % 2) == 0; }
 
