@@ -43,22 +43,9 @@ constexpr int SMEM_BYTES = SMEM_TILES + 1024;
 constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [key][d] with d contiguous
 
-// Of every HSWA_POLY_DEN element pairs, HSWA_POLY_NUM take 2^x on the FMA pipe instead of the MUFU.
-#ifndef HSWA_POLY_NUM
-#define HSWA_POLY_NUM 1
-#define HSWA_POLY_DEN 2
-#endif
-
-#ifdef HSWA_PROBE_TRACE
-__device__ long long hswa_trace[16 * 64];
-#define TRACE(slot, j) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (j) < 64) hswa_trace[(slot) * 64 + (j)] = clock64(); } while (0)
-#else
-#define TRACE(slot, j) do { } while (0)
-#endif
-
 // barrier indices
-enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9, BAR_PFULL = 11,
-       BAR_OFINAL = 13, NUM_BARS = 14 };
+enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9,
+       BAR_PFULL = 11 /* [Q tile][first / second half of each warp's columns] */, BAR_OFINAL = 15, NUM_BARS = 16 };
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -138,6 +125,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_st16p(uint32_t addr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};" ::"r"(r[0]),
+      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(addr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t* r) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};" ::"r"(r[0]), "r"(r[1]),
                "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(addr)
@@ -208,7 +203,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_PFULL + i), 8);  // one arrival per softmax warp
+      mbar_init(bar(BAR_PFULL + 2 * i), 8);  // one arrival per softmax warp
+      mbar_init(bar(BAR_PFULL + 2 * i + 1), 8);
     }
     mbar_init(bar(BAR_OFINAL), 1);
     mbar_fence_init();
@@ -304,13 +300,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         }
         tc_commit(bar(BAR_SFULL + i));
       };
-      auto issue_PV = [&](int i, int stage, bool first) {
+      // PV k-steps of one part: warps of column half h post keys 64 h + 32 part + [0, 32) = k-steps 4 h + 2 part + {0, 1}
+      auto issue_PV = [&](int i, int stage, int part, bool first) {
         tc_fence_after();
         const uint32_t aV = sbase + OFF_V + stage * TILE_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk)
+        for (int q = 0; q < 4; ++q) {
+          const int kk = (q >> 1) * 4 + part * 2 + (q & 1);
           tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, smem_desc(aV + kk * 2048, HALF_BYTES), IDESC_PV,
-                    !(first && kk == 0));
+                    !(first && part == 0 && q == 0));
+        }
       };
       if (ok) ok = mbar_wait(bar(BAR_KFULL + 0), 0);
       if (ok) {
@@ -323,24 +322,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         const bool more = j + 1 < n_tiles;
         ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + 0), j & 1);
         if (!ok) break;
-        TRACE(0, j);
-        issue_PV(0, stage, j == 0);
+        issue_PV(0, stage, 0, j == 0);
+        ok = mbar_wait(bar(BAR_PFULL + 1), j & 1);
+        if (!ok) break;
+        issue_PV(0, stage, 1, false);
         if (more) {
           ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
           if (!ok) break;
           issue_S(0, nstage);
         }
-        TRACE(1, j);
-        ok = mbar_wait(bar(BAR_PFULL + 1), j & 1);
+        ok = mbar_wait(bar(BAR_PFULL + 2), j & 1);
         if (!ok) break;
-        TRACE(2, j);
-        issue_PV(1, stage, j == 0);
+        issue_PV(1, stage, 0, j == 0);
+        ok = mbar_wait(bar(BAR_PFULL + 3), j & 1);
+        if (!ok) break;
+        issue_PV(1, stage, 1, false);
         tc_commit(bar(BAR_VEMPTY + stage));
         if (more) {
           issue_S(1, nstage);
           tc_commit(bar(BAR_KEMPTY + nstage));
         }
-        TRACE(3, j);
       }
       if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 20);
       tc_commit(bar(BAR_OFINAL));
@@ -364,13 +365,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + i), j & 1));  // warp-uniform: TMEM ops are warp-wide
-      if (lane == 0 && (warp & 7) == 0) TRACE(4 + 6 * i, j);
-#ifdef HSWA_PROBE_NO_SOFTMAX
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));
-      continue;
-#endif
       // visible column interval [lo, hi) of this row in this tile; ring tiles are decided per column
       int lo = 0, hi = BN;
       bool ring_tile = false, masked = false;
@@ -446,7 +440,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         }
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       }
-      if (lane == 0 && (warp & 7) == 0) TRACE(5 + 6 * i, j);
       xch[j & 1][i][half][rr] = mx;
       asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
       const float other = xch[j & 1][i][half ^ 1][rr];
@@ -455,7 +448,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         ok = false;
         break;
       }
-      if (lane == 0 && (warp & 7) == 0) TRACE(6 + 6 * i, j);
       mx = fmaxf(mx, other);
       const float mx_s = mx * M.scale_log2;
       if (j == 0) {
@@ -484,38 +476,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       float2 acc[4];
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[c] = make_float2(0.f, 0.f);
+      // Two parts of 32 keys each: the MMA warp starts the PV k-steps of a part as soon as all warps posted it,
+      // so half of the PV MMA overlaps the second part's exponentials.
 #pragma unroll
-      for (int k = 0; k < 32; ++k) {
-        const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
-        float2 e;
-        if ((k % HSWA_POLY_DEN) < HSWA_POLY_NUM) {
-          // 2^x on the FMA pipe: x = n + f with |f| <= 1/2 (magic-number rounding), cubic for 2^f (relative
-          // error 7.5e-5, far below bf16 rounding), n added into the exponent field.  The 16-lane MUFU would
-          // otherwise need 1024 clocks per 128 x 128 tile, about as long as the tile's four MMAs.
-          const float2 xc = make_float2(fmaxf(x.x, -126.f), fmaxf(x.y, -126.f));
-          const float2 t = __fadd2_rn(xc, make_float2(12582912.f, 12582912.f));
-          const float2 nf = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
-          const float2 f = __fadd2_rn(xc, make_float2(-nf.x, -nf.y));
-          float2 pl = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.242611125f, 0.242611125f));
-          pl = __ffma2_rn(pl, f, make_float2(0.693260968f, 0.693260968f));
-          pl = __ffma2_rn(pl, f, make_float2(0.999928057f, 0.999928057f));
-          e.x = __uint_as_float(__float_as_uint(pl.x) + (__float_as_uint(t.x) << 23));
-          e.y = __uint_as_float(__float_as_uint(pl.y) + (__float_as_uint(t.y) << 23));
-        } else {
-          e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+      for (int part = 0; part < 2; ++part) {
+#pragma unroll
+        for (int k = part * 16; k < part * 16 + 16; ++k) {
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
+          const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+          acc[k & 3] = __fadd2_rn(acc[k & 3], e);
+          v[k] = pack_bf16x2(e.x, e.y);
         }
-        acc[k & 3] = __fadd2_rn(acc[k & 3], e);
-        v[k] = pack_bf16x2(e.x, e.y);
+        tmem_st16p(tP + part * 16, v + part * 16);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_PFULL + 2 * i + part));  // 32 arrivals on one barrier word would serialise
       }
       const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
       l_run += (a01.x + a01.y) + (a23.x + a23.y);
-      if (lane == 0 && (warp & 7) == 0) TRACE(7 + 6 * i, j);
-      tmem_st32(tP, v);
-      tc_wait_st();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BAR_PFULL + i));  // 32 arrivals on one barrier word would serialise
-      if (lane == 0 && (warp & 7) == 0) TRACE(8 + 6 * i, j);
     }
     // ---- epilogue: O / l -> global ----
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFINAL), 0));
@@ -779,12 +758,6 @@ cudaError_t launch_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, cons
 }
 
 }  // namespace
-
-#ifdef HSWA_PROBE_TRACE
-extern "C" int hswa_debug_read_trace(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, hswa_trace, sizeof(long long) * 16 * 64);
-}
-#endif
 
 bool hswa_prefill_tc_supported(const ModelParams& m) { return m.D == 128 && m.P == 64 && (m.G % 2) == 0; }
 
