@@ -151,6 +151,9 @@ hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out) {
   h->num_sms = prop.multiProcessorCount;
   h->err = nullptr;
   h->encode_tiled = nullptr;
+  h->chain_stream = nullptr;
+  h->chain_ctx = nullptr;
+  h->chain_ok = 0;
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -193,6 +196,7 @@ size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max
 }
 
 hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, void* stream) {
+  if (h) h->chain_ok = 0;
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
   if (cudaSetDevice(h->device) != cudaSuccess) return HSWA_ERR_CUDA;
@@ -203,6 +207,7 @@ hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const h
 
 hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* k_new,
                            const void* v_new, void* stream) {
+  if (h) h->chain_ok = 0;
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
   if (b->batch == 0 || b->total_q == 0) return HSWA_OK;
@@ -264,14 +269,24 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
   CUtensorMap tm;
   st = make_pool_map(h, layer, &tm);
   if (st != HSWA_OK) return st;
-  if (hswa_launch_decode(h, tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  // A fused decode that directly follows another fused decode of the same step (same handle, stream and batch
+  // arrays) may start early: those kernels never write the batch arrays or another layer's pool.
+  const bool early = h->chain_ok && k_new != nullptr && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len;
+  h->chain_ok = 0;
+  if (hswa_launch_decode(h, tm, p, early, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (k_new != nullptr) {
+    h->chain_ok = 1;
+    h->chain_stream = stream;
+    h->chain_ctx = (const void*)b->ctx_len;
+  }
   return HSWA_OK;
 }
 
 hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,
                               const void* k_new, const void* v_new, int32_t fuse_append, void* out, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream) {
+  if (h) h->chain_ok = 0;
   (void)workspace;
   (void)workspace_bytes;
   hswa_status st = check_common(h, layer, b);
@@ -338,6 +353,7 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
 
 hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
                               const int32_t* q_indptr, void* stream) {
+  if (h) h->chain_ok = 0;
   if (!h || batch < 0) return HSWA_ERR_INVALID_ARG;
   if (batch == 0) return HSWA_OK;
   if (!ctx_len || !ring_head) return HSWA_ERR_INVALID_ARG;
@@ -347,6 +363,7 @@ hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, i
 }
 
 hswa_status hswa_get_async_error(hswa_handle* h, void* stream, int32_t info[4]) {
+  if (h) h->chain_ok = 0;
   if (!h || !info) return HSWA_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   if (cudaMemcpyAsync(info, h->err, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HSWA_ERR_CUDA;

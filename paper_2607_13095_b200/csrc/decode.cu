@@ -18,6 +18,12 @@ using namespace hswa_dev;
 
 constexpr int TK = 64;  // keys per pipeline stage
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while
+// the previous kernel on the stream is still running; everything it does before griddep_wait() must not depend
+// on that kernel.  Without the attribute both instructions do nothing.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 struct KeyRange {
   int is_swa;
   int span;   // Full: keys in this split; SWA: ring slots C
@@ -166,11 +172,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
       }
       __syncwarp();
     }
+    griddep_wait();  // this warp takes part in the output writes below
   } else {
     // ---------------- consumers ----------------
     const int cw = warp - 1;
     const int g_row = lane >> 2;  // head index used for the Q fragment (B operand column)
     uint32_t qf[KS][2];
+    // q, k_new, v_new may come from the previous kernel on the stream; the batch arrays and the cache that the
+    // producer warp is already streaming do not
+    griddep_wait();
+    griddep_launch_dependents();
     {
       const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
 #pragma unroll
@@ -381,6 +392,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
   const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   const ModelParams& M = p.m;
+  griddep_launch_dependents();  // the next attention kernel may start its cache loads now
   if (warp_global >= p.b.B * M.Hq) return;
   const int r = warp_global / M.Hq;
   const int64_t row = warp_global;
@@ -428,29 +440,38 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
 }
 
 template <int D, int P, int NS, int NW>
-cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, cudaStream_t s) {
+cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
   constexpr int SMEM = NS * STAGE_BYTES + 1024;
   static_assert(NW * 8 * D * 4 + NW * 64 <= NS * STAGE_BYTES, "merge scratch must fit the stage buffers");
   auto kern = decode_kernel<D, P, NS, NW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
-  dim3 grid(p.b.B, p.max_splits, p.m.Hkv);
-  kern<<<grid, (NW + 1) * 32, SMEM, s>>>(tm, p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.b.B, p.max_splits, p.m.Hkv);
+  cfg.blockDim = dim3((NW + 1) * 32, 1, 1);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, tm, p);
 }
 
 }  // namespace
 
-cudaError_t hswa_launch_decode(const hswa_handle*, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
+cudaError_t hswa_launch_decode(const hswa_handle*, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
+                               cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
   const int D = p.m.D, P = p.m.P;
-  if (D == 128 && P == 64) return launch_decode_t<128, 64, 3, 3>(tm_pool, p, s);
-  if (D == 128 && P == 32) return launch_decode_t<128, 32, 3, 3>(tm_pool, p, s);
-  if (D == 128 && P == 16) return launch_decode_t<128, 16, 3, 3>(tm_pool, p, s);
-  if (D == 64 && P == 64) return launch_decode_t<64, 64, 4, 3>(tm_pool, p, s);
-  if (D == 64 && P == 32) return launch_decode_t<64, 32, 4, 3>(tm_pool, p, s);
-  if (D == 64 && P == 16) return launch_decode_t<64, 16, 4, 3>(tm_pool, p, s);
+  if (D == 128 && P == 64) return launch_decode_t<128, 64, 3, 3>(tm_pool, p, early_start, s);
+  if (D == 128 && P == 32) return launch_decode_t<128, 32, 3, 3>(tm_pool, p, early_start, s);
+  if (D == 128 && P == 16) return launch_decode_t<128, 16, 3, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 64) return launch_decode_t<64, 64, 4, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 32) return launch_decode_t<64, 32, 4, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 16) return launch_decode_t<64, 16, 4, 3>(tm_pool, p, early_start, s);
   return cudaErrorInvalidValue;
 }
 

@@ -22,6 +22,11 @@ struct hswa_handle {
   int32_t num_sms;
   int32_t* err;  // device int32[4]
   hswa_encode_tiled_fn encode_tiled;
+  // Early-start bookkeeping: the last call through this handle was a fused decode on this stream and batch, so
+  // the next fused decode may overlap its prologue and cache loads with that kernel's tail.
+  void* chain_stream;
+  const void* chain_ctx;
+  int32_t chain_ok;
 };
 
 // Model constants every kernel needs.
@@ -89,7 +94,8 @@ struct PrefillParams {
 
 // Launchers implemented in the kernel translation units.
 cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s);
-cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s);
+cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
+                               cudaStream_t s);
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
 bool hswa_prefill_tc_supported(const ModelParams& m);

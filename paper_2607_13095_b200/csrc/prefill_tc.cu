@@ -666,35 +666,40 @@ prefill_swa_packed_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     float mx = -INFINITY, l_run = 0.f, m_use = 0.f;
     if (ok) {
       tc_fence_after();
+      // two passes over the N score columns in chunks of 32 (the last chunk is 16 or 32 wide)
+      constexpr int CH = (N + 31) / 32;
 #pragma unroll 1
-      for (int c = 0; c < N / 16; ++c) {
-        uint32_t v[16];
-        tmem_ld16(tS + c * 16, v);
+      for (int c = 0; c < CH; ++c) {
+        uint32_t v[32];
+        const bool wide = (c + 1) * 32 <= N;
+        if (wide) tmem_ld32(tS + c * 32, v); else tmem_ld16(tS + c * 32, v);
         tc_wait_ld();
+        const int cnt = wide ? 32 : 16;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int col = c * 16 + k;
-          if (col >= lo && col < hi) mx = fmaxf(mx, __uint_as_float(v[k]));
+        for (int k = 0; k < 32; ++k) {
+          const int col = c * 32 + k;
+          if (k < cnt && col >= lo && col < hi) mx = fmaxf(mx, __uint_as_float(v[k]));
         }
       }
       m_use = mx == -INFINITY ? 0.f : mx * M.scale_log2;
 #pragma unroll 1
-      for (int c = 0; c < N / 16; ++c) {
-        uint32_t v[16];
-        tmem_ld16(tS + c * 16, v);
+      for (int c = 0; c < CH; ++c) {
+        uint32_t v[32];
+        const bool wide = (c + 1) * 32 <= N;
+        if (wide) tmem_ld32(tS + c * 32, v); else tmem_ld16(tS + c * 32, v);
         tc_wait_ld();
-        uint32_t pk[8];
+        uint32_t pk[16];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int col = c * 16 + 2 * k;
+        for (int k = 0; k < 16; ++k) {
+          const int col = c * 32 + 2 * k;
           float p0 = fast_exp2(__uint_as_float(v[2 * k]) * M.scale_log2 - m_use);
           float p1 = fast_exp2(__uint_as_float(v[2 * k + 1]) * M.scale_log2 - m_use);
           p0 = (col >= lo && col < hi) ? p0 : 0.f;
           p1 = (col + 1 >= lo && col + 1 < hi) ? p1 : 0.f;
-          l_run += p0 + p1;
+          if (wide || k < 8) l_run += p0 + p1;
           pk[k] = pack_bf16x2(p0, p1);
         }
-        tmem_st8(tS + c * 8, pk);
+        if (wide) tmem_st16p(tS + c * 16, pk); else tmem_st8(tS + c * 16, pk);
       }
       tc_wait_st();
     } else if (lane == 0) {
