@@ -102,6 +102,9 @@ bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                    const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s);
 void hswa_prefill_packed_geometry(int G, int* tq, int* nkeys);
+cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                         const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int first_block,
+                                         cudaStream_t s);
 cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                            const PrefillParams& p, int first_tok, cudaStream_t s);
 cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,

@@ -762,6 +762,305 @@ cudaError_t launch_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, cons
   return cudaGetLastError();
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// SWA layers, GQA group of 8, tokens whose whole window lies inside the chunk: pipelined variant of the packed
+// kernel.  One block = 128 consecutive tokens of one (request, KV head).  The 256 chunk keys those tokens can
+// see are loaded once (K and V, 64 KB each); the block then walks eight sub-tiles of 16 tokens x 8 heads
+// (128 rows) against a 144-key slice of that buffer that slides by 16 rows per sub-tile.  Two softmax
+// warpgroups alternate sub-tiles, each with its own Q buffer and its own 256 TMEM columns (S in [0, 144), P
+// over its first 72 columns, O in [128, 256)), so the Q load, the S MMA, the softmax, the PV MMA and the
+// output of neighbouring sub-tiles overlap and K/V traffic is paid once per 128 tokens.
+namespace pipe {
+constexpr int SUB = 16;                         // tokens per sub-tile
+constexpr int NSUB = 8;                         // sub-tiles per block
+constexpr int N = 144;                          // keys per sub-tile (16 + 127, rounded up to 16)
+constexpr int KV_ROWS = 256;
+constexpr int KV_HALF = KV_ROWS * 128;          // bytes of one 64-element half
+constexpr int KV_BYTES = 2 * KV_HALF;           // 64 KB
+constexpr int QBUF = 3;                         // Q tiles in flight; a tile's buffer later stages its output
+constexpr int OFF_Q = 0, OFF_K = QBUF * TILE_BYTES, OFF_V = OFF_K + KV_BYTES;
+constexpr int SMEM = OFF_V + KV_BYTES + 1024;   // 225 KB
+constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+enum { B_K = 0, B_V = 1, B_QFULL = 2, B_QEMPTY = 5, B_SFULL = 8, B_PFULL = 10, B_OFULL = 12, B_OFREE = 14, NBARS = 16 };
+}  // namespace pipe
+
+__global__ void __launch_bounds__(320, 1)
+prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_out,
+                        const PrefillParams p, const int first_block, const int tma_out) {
+  using pipe::SUB; using pipe::NSUB; using pipe::N; using pipe::KV_HALF; using pipe::KV_BYTES;
+  using pipe::B_K; using pipe::B_V; using pipe::B_QFULL; using pipe::B_QEMPTY; using pipe::B_SFULL; using pipe::B_PFULL;
+  using pipe::B_OFULL; using pipe::B_OFREE; using pipe::NBARS; using pipe::QBUF;
+  constexpr int G = 8;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[NBARS];
+  __shared__ uint32_t tmem_base_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const ModelParams& M = p.m;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kh = blockIdx.x, r = blockIdx.z;
+  const int t0 = p.b.q_indptr[r];
+  const int n = p.b.q_indptr[r + 1] - t0;
+  const int i0 = (first_block + (int)blockIdx.y) * 128;  // first chunk-relative token of this block (>= 128)
+  if (i0 >= n) return;
+  if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;
+  const int n_sub = min(NSUB, (n - i0 + SUB - 1) / SUB);
+  const int key0 = i0 - 128;  // chunk-relative index of row 0 of the K/V buffer
+
+  auto bar = [&](int i) { return smem_u32(&bars[i]); };
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_K), 1);
+    mbar_init(bar(B_V), 1);
+    for (int q = 0; q < QBUF; ++q) {
+      mbar_init(bar(B_QFULL + q), 1);
+      mbar_init(bar(B_QEMPTY + q), 1);
+    }
+    for (int u = 0; u < 2; ++u) {
+      mbar_init(bar(B_SFULL + u), 1);
+      mbar_init(bar(B_PFULL + u), 4);
+      mbar_init(bar(B_OFULL + u), 1);
+      mbar_init(bar(B_OFREE + u), 4);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_slot;
+
+  if (warp == 8) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar(B_K), KV_BYTES);
+      for (int hf = 0; hf < 2; ++hf)
+        for (int rb = 0; rb < 2; ++rb)
+          tma_load_3d(sbase + pipe::OFF_K + hf * KV_HALF + rb * 128 * 128, &tm_k, bar(B_K), hf * 64, kh, t0 + key0 + rb * 128);
+      bool ok = true;
+      for (int s = 0; s < n_sub && ok; ++s) {
+        const int qb = s % QBUF;
+        if (s >= QBUF && !mbar_wait(bar(B_QEMPTY + qb), ((s / QBUF) - 1) & 1)) {
+          record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 60);
+          ok = false;
+          break;
+        }
+        mbar_arrive_expect_tx(bar(B_QFULL + qb), TILE_BYTES);
+        for (int hf = 0; hf < 2; ++hf)
+          tma_load_3d(sbase + pipe::OFF_Q + qb * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(B_QFULL + qb), hf * 64, kh * G, t0 + i0 + s * SUB);
+        if (s == 1 || n_sub == 1) {  // V is needed after the first softmax only: queue it behind the first Q tiles
+          mbar_arrive_expect_tx(bar(B_V), KV_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            for (int rb = 0; rb < 2; ++rb)
+              tma_load_3d(sbase + pipe::OFF_V + hf * KV_HALF + rb * 128 * 128, &tm_v, bar(B_V), hf * 64, kh, t0 + key0 + rb * 128);
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ======================= MMA issuer =======================
+    if (lane == 0) {
+      auto issue_S = [&](int s) {
+        const int u = s & 1;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t aq = sbase + pipe::OFF_Q + (s % QBUF) * TILE_BYTES + (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+          const uint32_t ak = sbase + pipe::OFF_K + (ks >> 2) * KV_HALF + s * SUB * 128 + (ks & 3) * 32;
+          tc_mma_ss(tmem + u * 256, smem_desc(aq, 16), smem_desc(ak, 16), pipe::IDESC_S, ks > 0);
+        }
+        tc_commit(bar(B_SFULL + u));
+      };
+      auto issue_PV = [&](int s) {
+        const int u = s & 1;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < N / 16; ++kk)
+          tc_mma_ts(tmem + u * 256 + 128, tmem + u * 256 + kk * 8, smem_desc(sbase + pipe::OFF_V + s * SUB * 128 + kk * 2048, KV_HALF),
+                    IDESC_PV, kk > 0);
+        tc_commit(bar(B_OFULL + u));
+      };
+      bool ok = mbar_wait(bar(B_K), 0);
+      for (int s = 0; s < 2 && s < n_sub && ok; ++s) {
+        ok = mbar_wait(bar(B_QFULL + s), 0);
+        if (ok) issue_S(s);
+      }
+      if (ok) ok = mbar_wait(bar(B_V), 0);
+      for (int s0 = 0; s0 < n_sub && ok; s0 += 2) {
+        for (int s = s0; s < s0 + 2 && s < n_sub && ok; ++s) {
+          ok = mbar_wait(bar(B_PFULL + (s & 1)), (s >> 1) & 1);
+          if (ok) issue_PV(s);
+        }
+        for (int s = s0 + 2; s < s0 + 4 && s < n_sub && ok; ++s) {
+          // the buffer's previous output must have left TMEM, and the next Q tile must have landed
+          ok = mbar_wait(bar(B_OFREE + (s & 1)), ((s >> 1) - 1) & 1) && mbar_wait(bar(B_QFULL + s % QBUF), (s / QBUF) & 1);
+          if (ok) issue_S(s);
+        }
+      }
+      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 61);
+    }
+  } else {
+    // ======================= softmax warpgroups: warps 0-3 take even sub-tiles, 4-7 odd =======================
+    const int u = warp >> 2;
+    const int rr = (warp & 3) * 32 + lane;  // row = TMEM lane
+    const int tl = rr / G, g = rr % G;      // token within the sub-tile, head within the group
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_addr + u * 256, tO = tS + 128;
+    const int lo = tl + 129 - M.W, hi = tl + 129;  // visible key columns [lo, hi) of the 144-key slice
+    for (int s = u; s < n_sub; s += 2) {
+      const uint32_t par = (s >> 1) & 1;
+      bool ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SFULL + u), par));
+      float l_run = 0.f, m_use = 0.f;
+      if (ok) {
+        tc_fence_after();
+        // the row's 144 scores in one round trip to TMEM; only columns [0, 32) and [128, 144) can be masked
+        uint32_t v[N];
+        tmem_ld32(tS, v);
+        tmem_ld32(tS + 32, v + 32);
+        tmem_ld32(tS + 64, v + 64);
+        tmem_ld32(tS + 96, v + 96);
+        tmem_ld16(tS + 128, v + 128);
+        tc_wait_ld();
+        {
+          const uint32_t head_mask = lo >= 32 ? 0u : (0xffffffffu << (lo < 0 ? 0 : lo));     // columns 0-31: col >= lo
+          const int t = hi - 128;                                                               // columns 128-143: col < hi
+          const uint32_t tail_mask = t >= 16 ? 0xffffu : (t <= 0 ? 0u : ((1u << t) - 1u));
+#pragma unroll
+          for (int k = 0; k < 32; ++k)
+            if (!((head_mask >> k) & 1u)) v[k] = 0xff800000u;
+#pragma unroll
+          for (int k = 0; k < 16; ++k)
+            if (!((tail_mask >> k) & 1u)) v[128 + k] = 0xff800000u;
+        }
+        float mx4[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mx4[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+#pragma unroll
+        for (int k = 8; k < N; k += 8) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mx4[c] = max3(mx4[c], __uint_as_float(v[k + 2 * c]), __uint_as_float(v[k + 2 * c + 1]));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        m_use = mx == -INFINITY ? 0.f : mx * M.scale_log2;
+        const float2 sc2 = make_float2(M.scale_log2, M.scale_log2), nm2 = make_float2(-m_use, -m_use);
+        float2 acc[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[c] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < N / 2; ++k) {
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
+          const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));  // masked columns: 2^(-inf) = 0
+          acc[k & 3] = __fadd2_rn(acc[k & 3], e);
+          v[k] = pack_bf16x2(e.x, e.y);
+        }
+        const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
+        l_run = (a01.x + a01.y) + (a23.x + a23.y);
+        tmem_st32(tS, v);
+        tmem_st32(tS + 32, v + 32);
+        tmem_st8(tS + 64, v + 64);
+        tc_wait_st();
+      } else if (lane == 0) {
+        record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 62);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_PFULL + u));
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OFULL + u), par));
+      tc_fence_after();
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      const int tok = i0 + s * SUB + tl;
+      const bool row_ok = ok && tok < n;
+      const int64_t orow = (int64_t)(t0 + tok) * M.Hq + kh * G + g;
+      const int qb = s % QBUF;
+      // Full sub-tiles with bf16 output leave through shared memory (the sub-tile's own Q buffer, idle since its
+      // S MMA) and one TMA tensor store; a row-per-thread global store would touch 32 scattered sectors per
+      // instruction.  Ragged tails and fp32 output use plain stores.
+      const bool staged = tma_out && ok && (i0 + s * SUB + SUB <= n);
+      uint8_t* stage = smem + pipe::OFF_Q + qb * TILE_BYTES;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t w[32];
+        tmem_ld32(tO + c4 * 32, w);
+        tc_wait_ld();
+        if (staged) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            uint4 x;
+            x.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
+            x.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
+            x.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
+            x.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
+            const int chunk = c4 * 4 + k;  // 16-byte chunk of the 256-byte row
+            *reinterpret_cast<uint4*>(stage + (chunk >> 3) * HALF_BYTES + swz128(rr, chunk & 7)) = x;
+          }
+        } else if (row_ok) {
+          if (M.out_fp32) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
+                                   __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + c4 * 32);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              uint4 x;
+              x.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
+              x.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
+              x.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
+              x.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
+              dst[k] = x;
+            }
+          }
+        }
+      }
+      if (row_ok && p.lse) p.lse[orow] = l_run > 0.f ? (m_use + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+      // the accumulator has been read out: the MMA warp may reuse this TMEM buffer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_OFREE + u));
+      // hand the staged tile to TMA (or just release the Q buffer)
+      if (staged) fence_proxy_async_smem();
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + u) : "memory");
+      if ((warp & 3) == 0 && lane == 0) {
+        if (staged) {
+          for (int hf = 0; hf < 2; ++hf)
+            asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_out),
+                         "r"(sbase + pipe::OFF_Q + qb * TILE_BYTES + hf * HALF_BYTES), "r"(hf * 64), "r"(kh * G),
+                         "r"(t0 + i0 + s * SUB)
+                         : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory has been read: the buffer is free
+        }
+        mbar_arrive(bar(B_QEMPTY + qb));
+      }
+    }
+    if ((warp & 3) == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores have landed
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+cudaError_t launch_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_out,
+                        int tma_out, const PrefillParams& p, int first_block, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(prefill_swa_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe::SMEM);
+  if (e != cudaSuccess) return e;
+  const int blocks = (p.max_q_len + 127) / 128 - first_block;
+  if (blocks <= 0) return cudaSuccess;
+  dim3 grid(p.m.Hkv, blocks, p.b.B);
+  prefill_swa_pipe_kernel<<<grid, 320, pipe::SMEM, s>>>(tm_q, tm_k, tm_v, tm_out, p, first_block, tma_out);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool hswa_prefill_tc_supported(const ModelParams& m) { return m.D == 128 && m.P == 64 && (m.G % 2) == 0; }
@@ -780,6 +1079,17 @@ cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtens
   if (p.m.G == 8) return launch_packed<8>(tm_q, tm_k, tm_v, p, first_tok, s);
   if (p.m.G == 4) return launch_packed<4>(tm_q, tm_k, tm_v, p, first_tok, s);
   return cudaErrorInvalidValue;
+}
+
+// Pipelined SWA kernel (GQA group of 8): blocks of 128 tokens starting at block `first_block`; tm_q has box
+// {64, 8 heads, 16 tokens}, tm_k / tm_v have box {64, 1, 128 rows}; tm_out is tm_q's twin over a bf16 output
+// tensor (used when tma_out != 0).
+cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                         const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int first_block,
+                                         cudaStream_t s) {
+  if (p.m.G != 8) return cudaErrorInvalidValue;
+  if (p.b.B == 0) return cudaSuccess;
+  return launch_pipe(tm_q, tm_k, tm_v, tm_out, tma_out, p, first_block, s);
 }
 
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
