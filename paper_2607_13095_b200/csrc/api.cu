@@ -221,6 +221,7 @@ hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_b
   p.k_new = static_cast<const __nv_bfloat16*>(k_new);
   p.v_new = static_cast<const __nv_bfloat16*>(v_new);
   p.total_q = b->total_q;
+  p.max_q_len = b->max_q_len;
   return hswa_launch_append(p, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
@@ -355,6 +356,7 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
     a.k_new = p.k_new;
     a.v_new = p.v_new;
     a.total_q = p.total_q;
+    a.max_q_len = p.max_q_len;
     if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   }
   return HSWA_OK;

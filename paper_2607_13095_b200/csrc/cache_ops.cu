@@ -16,7 +16,7 @@ __device__ __forceinline__ int find_request(const BatchParams& b, int t) {
   return lo;
 }
 
-// One thread moves one 16-byte chunk of one (token, K|V, head) row.
+// One thread moves one 16-byte chunk of one (token, K|V, head) row of a Full layer.
 __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
   const ModelParams& M = p.m;
   const int chunks_per_row = M.D / 8;
@@ -33,24 +33,40 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
 
   const int r = find_request(p.b, t);
   const int t0 = p.b.q_indptr ? p.b.q_indptr[r] : r;
-  const int n = p.b.q_indptr ? p.b.q_indptr[r + 1] - t0 : 1;
-  const int i = t - t0;
-  const int ctx = p.b.ctx_len[r];
-  int page, slot;
-  if (!p.is_swa) {
-    const int pos = ctx + i;
-    const int blk = pos / M.P;
-    if (blk >= p.b.max_blocks) return;
-    page = p.b.block_table[(int64_t)r * p.b.max_blocks + blk];
-    slot = pos % M.P;
-  } else {
-    if (n - i > M.C) return;  // overwritten later in this same step: only the last C tokens survive
-    const int s = math_mod(p.b.ring_head[r] + i, M.C);
-    page = p.b.ring_table[(int64_t)r * M.R + s / M.P];
-    slot = s % M.P;
-  }
+  const int pos = p.b.ctx_len[r] + (t - t0);
+  const int blk = pos / M.P;
+  if (blk >= p.b.max_blocks) return;
+  const int page = p.b.block_table[(int64_t)r * p.b.max_blocks + blk];
+  const int slot = pos % M.P;
   if (page < 0 || page >= p.num_pages) return;
   const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)t * M.Hkv + kh) * M.D + ch * 8;
+  __nv_bfloat16* dst = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + slot) * M.D + ch * 8;
+  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+}
+
+// SWA layer: only the last min(n, C) tokens of a request survive on its ring (later writes win), so the grid
+// covers C tokens per request (blockIdx.y = request) instead of the whole chunk.
+__global__ void __launch_bounds__(256) append_ring_kernel(const AppendParams p) {
+  const ModelParams& M = p.m;
+  const int chunks_per_row = M.D / 8;
+  const int chunks_per_tok = 2 * M.Hkv * chunks_per_row;
+  const int r = blockIdx.y;
+  const int t0 = p.b.q_indptr ? p.b.q_indptr[r] : r;
+  const int n = p.b.q_indptr ? p.b.q_indptr[r + 1] - t0 : 1;
+  const int keep = min(n, M.C);
+  const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= keep * chunks_per_tok) return;
+  const int i = n - keep + gid / chunks_per_tok;  // chunk-relative token
+  int c = gid % chunks_per_tok;
+  const int kv = c / (M.Hkv * chunks_per_row);
+  c -= kv * M.Hkv * chunks_per_row;
+  const int kh = c / chunks_per_row;
+  const int ch = c % chunks_per_row;
+  const int s = math_mod(p.b.ring_head[r] + (i % M.C), M.C);
+  const int page = p.b.ring_table[(int64_t)r * M.R + s / M.P];
+  const int slot = s % M.P;
+  if (page < 0 || page >= p.num_pages) return;
+  const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)(t0 + i) * M.Hkv + kh) * M.D + ch * 8;
   __nv_bfloat16* dst = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + slot) * M.D + ch * 8;
   *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
 }
@@ -99,10 +115,17 @@ __global__ void __launch_bounds__(128) validate_kernel(ModelParams M, BatchParam
 }  // namespace
 
 cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s) {
-  const int64_t total = (int64_t)p.total_q * 2 * p.m.Hkv * (p.m.D / 8);
-  if (total == 0) return cudaSuccess;
-  const int64_t blocks = (total + 255) / 256;
-  append_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
+  const int chunks_per_tok = 2 * p.m.Hkv * (p.m.D / 8);
+  if (p.total_q == 0 || p.b.B == 0) return cudaSuccess;
+  if (p.is_swa) {
+    const int per_req = min(p.max_q_len, p.m.C) * chunks_per_tok;
+    if (per_req == 0) return cudaSuccess;
+    dim3 grid((per_req + 255) / 256, p.b.B);
+    append_ring_kernel<<<grid, 256, 0, s>>>(p);
+  } else {
+    const int64_t total = (int64_t)p.total_q * chunks_per_tok;
+    append_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(p);
+  }
   return cudaGetLastError();
 }
 

@@ -74,6 +74,7 @@ struct AppendParams {
   const __nv_bfloat16* k_new;
   const __nv_bfloat16* v_new;
   int32_t total_q;
+  int32_t max_q_len;  // host-known bound of new tokens per request
 };
 
 struct PrefillParams {

@@ -778,20 +778,22 @@ constexpr int N = 144;                          // keys per sub-tile (16 + 127, 
 constexpr int KV_ROWS = 256;
 constexpr int KV_HALF = KV_ROWS * 128;          // bytes of one 64-element half
 constexpr int KV_BYTES = 2 * KV_HALF;           // 64 KB
-constexpr int QBUF = 3;                         // Q tiles in flight; a tile's buffer later stages its output
-constexpr int OFF_Q = 0, OFF_K = QBUF * TILE_BYTES, OFF_V = OFF_K + KV_BYTES;
-constexpr int SMEM = OFF_V + KV_BYTES + 1024;   // 225 KB
+constexpr int QBUF = 2;                         // Q tiles in flight (a buffer is free as soon as its S MMA has run)
+constexpr int OFF_Q = 0, OFF_K = QBUF * TILE_BYTES, OFF_V = OFF_K + KV_BYTES, OFF_STAGE = OFF_V + KV_BYTES;
+constexpr int SMEM = OFF_STAGE + TILE_BYTES + 1024;   // 225 KB: Q 64, K 64, V 64, output staging 32
 constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-enum { B_K = 0, B_V = 1, B_QFULL = 2, B_QEMPTY = 5, B_SFULL = 8, B_PFULL = 10, B_OFULL = 12, B_OFREE = 14, NBARS = 16 };
+enum { B_K = 0, B_V = 1, B_QFULL = 2, B_QEMPTY = 4, B_SFULL = 6, B_PFULL = 8, B_OFULL = 10, B_OFREE = 12, B_STAGED = 14,
+       B_STGFREE = 15, NBARS = 16 };
+constexpr int THREADS = 352;                    // 8 softmax warps + producer + MMA issuer + output store warp
 }  // namespace pipe
 
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(pipe::THREADS, 1)
 prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                         const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_out,
                         const PrefillParams p, const int first_block, const int tma_out) {
   using pipe::SUB; using pipe::NSUB; using pipe::N; using pipe::KV_HALF; using pipe::KV_BYTES;
   using pipe::B_K; using pipe::B_V; using pipe::B_QFULL; using pipe::B_QEMPTY; using pipe::B_SFULL; using pipe::B_PFULL;
-  using pipe::B_OFULL; using pipe::B_OFREE; using pipe::NBARS; using pipe::QBUF;
+  using pipe::B_OFULL; using pipe::B_OFREE; using pipe::B_STAGED; using pipe::B_STGFREE; using pipe::NBARS; using pipe::QBUF;
   constexpr int G = 8;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[NBARS];
@@ -814,6 +816,8 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   if (threadIdx.x == 0) {
     mbar_init(bar(B_K), 1);
     mbar_init(bar(B_V), 1);
+    mbar_init(bar(B_STAGED), 4);
+    mbar_init(bar(B_STGFREE), 1);
     for (int q = 0; q < QBUF; ++q) {
       mbar_init(bar(B_QFULL + q), 1);
       mbar_init(bar(B_QEMPTY + q), 1);
@@ -875,6 +879,7 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           tc_mma_ss(tmem + u * 256, smem_desc(aq, 16), smem_desc(ak, 16), pipe::IDESC_S, ks > 0);
         }
         tc_commit(bar(B_SFULL + u));
+        tc_commit(bar(B_QEMPTY + s % QBUF));  // Q(s) has been consumed once these MMAs are done
       };
       auto issue_PV = [&](int s) {
         const int u = s & 1;
@@ -885,24 +890,61 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
                     IDESC_PV, kk > 0);
         tc_commit(bar(B_OFULL + u));
       };
+      // Issue whichever MMA group has its inputs first: S(s) needs Q(s) in shared memory and, from the third
+      // sub-tile on, the output of S(s - 2)'s TMEM buffer read out; PV(s) needs P(s) (and V).  Sub-tiles of the
+      // two warpgroups interleave, so neither waits behind the other's hand-off.
       bool ok = mbar_wait(bar(B_K), 0);
-      for (int s = 0; s < 2 && s < n_sub && ok; ++s) {
-        ok = mbar_wait(bar(B_QFULL + s), 0);
-        if (ok) issue_S(s);
-      }
-      if (ok) ok = mbar_wait(bar(B_V), 0);
-      for (int s0 = 0; s0 < n_sub && ok; s0 += 2) {
-        for (int s = s0; s < s0 + 2 && s < n_sub && ok; ++s) {
-          ok = mbar_wait(bar(B_PFULL + (s & 1)), (s >> 1) & 1);
-          if (ok) issue_PV(s);
+      int next_s = 0, next_pv = 0;
+      bool v_ready = false;
+      long long t_start = clock64();
+      while (ok && next_pv < n_sub) {
+        bool progress = false;
+        if (next_s < n_sub) {
+          const int s = next_s;
+          const bool free_ok = s < 2 || mbar_try_wait(bar(B_OFREE + (s & 1)), ((s >> 1) - 1) & 1);
+          if (free_ok && mbar_try_wait(bar(B_QFULL + s % QBUF), (s / QBUF) & 1)) {
+            issue_S(s);
+            ++next_s;
+            progress = true;
+          }
         }
-        for (int s = s0 + 2; s < s0 + 4 && s < n_sub && ok; ++s) {
-          // the buffer's previous output must have left TMEM, and the next Q tile must have landed
-          ok = mbar_wait(bar(B_OFREE + (s & 1)), ((s >> 1) - 1) & 1) && mbar_wait(bar(B_QFULL + s % QBUF), (s / QBUF) & 1);
-          if (ok) issue_S(s);
+        if (next_pv < next_s && mbar_try_wait(bar(B_PFULL + (next_pv & 1)), (next_pv >> 1) & 1)) {
+          if (!v_ready) {
+            ok = mbar_wait(bar(B_V), 0);
+            v_ready = true;
+          }
+          if (ok) issue_PV(next_pv);
+          ++next_pv;
+          progress = true;
+        }
+        if (progress) {
+          t_start = clock64();
+        } else if (clock64() - t_start > 4000000000LL) {
+          ok = false;
         }
       }
       if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 61);
+    }
+  } else if (warp == 10) {
+    // ======================= output store warp =======================
+    // Takes each staged output tile to global memory with one TMA tensor store per half and frees the staging
+    // buffer once shared memory has been read, so no softmax thread waits for a store.
+    if (lane == 0 && tma_out) {
+      bool ok = true;
+      for (int s = 0; s < n_sub && ok; ++s) {
+        if (i0 + s * SUB + SUB > n) break;  // a ragged last sub-tile is stored directly by its warpgroup
+        ok = mbar_wait(bar(B_STAGED), s & 1);
+        if (!ok) break;
+        for (int hf = 0; hf < 2; ++hf)
+          asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_out),
+                       "r"(sbase + pipe::OFF_STAGE + hf * HALF_BYTES), "r"(hf * 64), "r"(kh * G), "r"(t0 + i0 + s * SUB)
+                       : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory has been read
+        mbar_arrive(bar(B_STGFREE));
+      }
+      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 63);
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores have landed
     }
   } else {
     // ======================= softmax warpgroups: warps 0-3 take even sub-tiles, 4-7 odd =======================
@@ -977,38 +1019,46 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       const bool row_ok = ok && tok < n;
       const int64_t orow = (int64_t)(t0 + tok) * M.Hq + kh * G + g;
       const int qb = s % QBUF;
-      // Full sub-tiles with bf16 output leave through shared memory (the sub-tile's own Q buffer, idle since its
-      // S MMA) and one TMA tensor store; a row-per-thread global store would touch 32 scattered sectors per
+      // Full sub-tiles with bf16 output leave through a shared-memory staging tile and one TMA tensor store; a row-per-thread global store would touch 32 scattered sectors per
       // instruction.  Ragged tails and fp32 output use plain stores.
       const bool staged = tma_out && ok && (i0 + s * SUB + SUB <= n);
-      uint8_t* stage = smem + pipe::OFF_Q + qb * TILE_BYTES;
-#pragma unroll 1
-      for (int c4 = 0; c4 < 4; ++c4) {
-        uint32_t w[32];
-        tmem_ld32(tO + c4 * 32, w);
+      uint8_t* stage = smem + pipe::OFF_STAGE;
+      {
+        uint32_t w[128];  // the whole accumulator row in one round trip
+        tmem_ld32(tO, w);
+        tmem_ld32(tO + 32, w + 32);
+        tmem_ld32(tO + 64, w + 64);
+        tmem_ld32(tO + 96, w + 96);
         tc_wait_ld();
+        // the accumulator has been read out: the MMA warp may reuse this TMEM buffer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_OFREE + u));
         if (staged) {
+          // sub-tiles use the single staging tile in order: wait until the previous one's store has read it
+          if (s > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(B_STGFREE), (s - 1) & 1))) {
+            if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 64);
+          }
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
+          for (int chunk = 0; chunk < 16; ++chunk) {  // 16-byte chunks of the 256-byte bf16 row
             uint4 x;
-            x.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
-            x.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
-            x.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
-            x.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
-            const int chunk = c4 * 4 + k;  // 16-byte chunk of the 256-byte row
+            x.x = pack_bf16x2(__uint_as_float(w[8 * chunk]) * inv, __uint_as_float(w[8 * chunk + 1]) * inv);
+            x.y = pack_bf16x2(__uint_as_float(w[8 * chunk + 2]) * inv, __uint_as_float(w[8 * chunk + 3]) * inv);
+            x.z = pack_bf16x2(__uint_as_float(w[8 * chunk + 4]) * inv, __uint_as_float(w[8 * chunk + 5]) * inv);
+            x.w = pack_bf16x2(__uint_as_float(w[8 * chunk + 6]) * inv, __uint_as_float(w[8 * chunk + 7]) * inv);
             *reinterpret_cast<uint4*>(stage + (chunk >> 3) * HALF_BYTES + swz128(rr, chunk & 7)) = x;
           }
         } else if (row_ok) {
           if (M.out_fp32) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + c4 * 32);
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
+            for (int k = 0; k < 32; ++k)
               dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
                                    __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
           } else {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + c4 * 32);
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < 16; ++k) {
               uint4 x;
               x.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
               x.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
@@ -1020,27 +1070,13 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         }
       }
       if (row_ok && p.lse) p.lse[orow] = l_run > 0.f ? (m_use + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-      // the accumulator has been read out: the MMA warp may reuse this TMEM buffer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_OFREE + u));
-      // hand the staged tile to TMA (or just release the Q buffer)
-      if (staged) fence_proxy_async_smem();
-      asm volatile("bar.sync %0, 128;" ::"r"(1 + u) : "memory");
-      if ((warp & 3) == 0 && lane == 0) {
-        if (staged) {
-          for (int hf = 0; hf < 2; ++hf)
-            asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_out),
-                         "r"(sbase + pipe::OFF_Q + qb * TILE_BYTES + hf * HALF_BYTES), "r"(hf * 64), "r"(kh * G),
-                         "r"(t0 + i0 + s * SUB)
-                         : "memory");
-          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory has been read: the buffer is free
-        }
-        mbar_arrive(bar(B_QEMPTY + qb));
+      // hand the staged tile to the store warp
+      if (staged) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_STAGED));
       }
     }
-    if ((warp & 3) == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores have landed
   }
   tc_fence_before();
   __syncthreads();
@@ -1057,7 +1093,7 @@ cudaError_t launch_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const 
   const int blocks = (p.max_q_len + 127) / 128 - first_block;
   if (blocks <= 0) return cudaSuccess;
   dim3 grid(p.m.Hkv, blocks, p.b.B);
-  prefill_swa_pipe_kernel<<<grid, 320, pipe::SMEM, s>>>(tm_q, tm_k, tm_v, tm_out, p, first_block, tma_out);
+  prefill_swa_pipe_kernel<<<grid, pipe::THREADS, pipe::SMEM, s>>>(tm_q, tm_k, tm_v, tm_out, p, first_block, tma_out);
   return cudaGetLastError();
 }
 
