@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
+    ap.add_argument("--cascade", action="store_true", help="cfg4: use hswa_decode_attn_shared_prefix on the shared prefix")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill block reported under 'extra'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -131,7 +132,8 @@ class ClockSampler:
 class DecodeBench:
     """Device-resident state of a decode workload and one-step runner."""
 
-    def __init__(self, w, total_steps, device):
+    def __init__(self, w, total_steps, device, cascade=False):
+        self.shared_prefix = w.tables.shared_prefix_pages * w.dims.page_size if cascade else 0
         import torch
         from paper_2607_13095_b200 import binding as hb
         from paper_2607_13095_b200 import workloads as wl
@@ -165,7 +167,7 @@ class DecodeBench:
         ws_bytes = hb.hswa_workspace_bytes(self.h, B, B, self.max_ctx)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=device)
         self.full_idx = [i for i, s in enumerate(w.layer_is_swa) if not s]
-        self.launches_per_step = sum(1 if s else 2 for s in w.layer_is_swa) + 1
+        self.launches_per_step = sum(1 if s else (3 if self.shared_prefix else 2) for s in w.layer_is_swa) + 1
 
     def reset(self):
         self.ctx.copy_(self.ctx0)
@@ -177,8 +179,12 @@ class DecodeBench:
             timed = events is not None and i == self.full_idx[0]
             if timed:
                 events[0].record()
-            hb.hswa_decode_attn(self.h, layer, self.batch, self.q[i], self.k_new[i], self.v_new[i], self.out[i], None,
-                                self.ws)
+            if self.shared_prefix:
+                hb.hswa_decode_attn_shared_prefix(self.h, layer, self.batch, self.shared_prefix, self.q[i], self.k_new[i],
+                                                  self.v_new[i], self.out[i], None, self.ws)
+            else:
+                hb.hswa_decode_attn(self.h, layer, self.batch, self.q[i], self.k_new[i], self.v_new[i], self.out[i], None,
+                                    self.ws)
             if timed:
                 events[1].record()
         hb.hswa_step_advance(self.h, self.t.batch, self.ctx, self.head, None)
@@ -442,7 +448,7 @@ def main():
         return
     w = make_workload(args.workload, seed_offset=rank, layers=args.layers, batch=args.batch)
     total_steps = args.steps + args.warmup
-    bench = DecodeBench(w, 2 * total_steps + 8, device)
+    bench = DecodeBench(w, 2 * total_steps + 8, device, cascade=args.cascade)
     t, d = bench.t, w.dims
 
     def barrier():
@@ -530,7 +536,8 @@ def main():
         "config": {"workload": w.name, "layers": len(w.layer_is_swa), "swa_layers": int(sum(w.layer_is_swa)),
                    "batch": t.batch, "num_q_heads": d.num_q_heads, "num_kv_heads": d.num_kv_heads,
                    "head_dim": d.head_dim, "page_size": d.page_size, "window": d.window,
-                   "ctx_sum": int(t.ctx_len.sum()), "l2": "inputs larger than L2 (Full-layer KV streamed per step "
+                   "ctx_sum": int(t.ctx_len.sum()), "shared_prefix_tokens": t.shared_prefix_pages * d.page_size,
+                   "cascade": bool(args.cascade), "l2": "inputs larger than L2 (Full-layer KV streamed per step "
                    "exceeds 126 MB and evicts the SWA rings between reuses)", "out_dtype": "bf16"},
         "step_gbs": step_bytes / (ms_step * 1e-3) / 1e9 * world,
         "step_frac_of_measured_hbm": step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -132,6 +132,22 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
                              const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, void* stream);
 
+/* Cascade decode for batches whose requests all share a cached prefix (paper Sec. 3.1.3: equal token prefixes
+ * share KV pages; Sec. 3.1.4: multi-user shared system prompts).  Same arguments and results as
+ * hswa_decode_attn plus shared_prefix_len: the caller (its prefix tree) guarantees that the first
+ * shared_prefix_len tokens of EVERY request in the batch map to the same physical pages, i.e. the leading
+ * shared_prefix_len / P block-table entries are identical across requests, that shared_prefix_len is a multiple
+ * of P and that shared_prefix_len <= ctx_len[r] for all r.  On Full layers the shared keys are then attended
+ * once per group of requests as a dense tensor-core problem (rows = requests x heads) instead of being streamed
+ * once per request, and merged with the per-request suffixes in the split combine.  SWA layers, shapes the
+ * tensor-core stage does not cover (it needs D = 128, P = 64, G = 8) and prefixes shorter than 128 tokens take
+ * the hswa_decode_attn path; results are the same up to fp32 rounding order.  shared_prefix_len = 0 is
+ * hswa_decode_attn.  Not a multiple of P, negative or above max_ctx_len: HSWA_ERR_INVALID_ARG. */
+hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch,
+                                           int32_t shared_prefix_len, const void* q, const void* k_new,
+                                           const void* v_new, void* out, float* lse, void* workspace,
+                                           size_t workspace_bytes, void* stream);
+
 /* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart of this
  * call; it exists for deployment reasons only.)
  * Same arguments, results and errors as hswa_decode_attn, minus the workspace: the split-K partials go to a

@@ -189,7 +189,9 @@ size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max
   const size_t kv = (size_t)max_ctx_len + 1;
   const size_t long_splits = (kv + kMaxSplitLen - 1) / kMaxSplitLen + 2;
   const size_t want = 4 * (size_t)h->num_sms;
-  const size_t row_splits = (size_t)h->cfg.num_q_heads * max_batch * long_splits + 2 * want * h->group;
+  // (+ the shared-prefix slices of cascade decode: at most num_sms / (groups of 32 requests x Hkv) per row)
+  const size_t row_splits = (size_t)h->cfg.num_q_heads * max_batch * long_splits + 2 * want * h->group +
+                            (size_t)32 * h->group * h->num_sms;
   const size_t o_bytes = row_splits * h->cfg.head_dim * sizeof(float);
   const size_t ml_bytes = row_splits * sizeof(float2);
   return ((o_bytes + 255) & ~size_t(255)) + ((ml_bytes + 255) & ~size_t(255));
@@ -225,9 +227,9 @@ hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_b
   return hswa_launch_append(p, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
-hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,
-                             const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, int32_t shared_prefix_len,
+                               const void* q, const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
+                               size_t workspace_bytes, void* stream) {
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
   if (b->q_indptr != nullptr) return HSWA_ERR_INVALID_ARG;
@@ -250,13 +252,33 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
   p.err = h->err;
   p.part_o = nullptr;
   p.part_ml = nullptr;
+  p.k_start = 0;
+  p.split_base = 0;
+  // Cascade decode: the shared prefix is attended once per group of requests on the tensor cores, the
+  // per-request suffixes by the streaming kernel; both leave partials for the combine.
+  const bool cascade = !layer->is_swa && shared_prefix_len >= 128 && h->cfg.head_dim == 128 && h->cfg.page_size == 64 &&
+                       h->group == 8;
+  int prefix_slices = 0, prefix_tps = 0;
   if (layer->is_swa) {
     p.split_len = ((h->ring_slots + 63) / 64) * 64;
     p.max_splits = 1;
+    p.grid_splits = 1;
   } else {
-    p.split_len = plan_split_len(h, b->batch, b->max_ctx_len);
-    p.max_splits = plan_max_splits(p.split_len, b->max_ctx_len);
-    if (p.max_splits > 65535) return HSWA_ERR_UNSUPPORTED;
+    if (cascade) {
+      const int tiles = (shared_prefix_len + 127) / 128;
+      const int base = ((b->batch + 31) / 32) * h->cfg.num_kv_heads;
+      int want = h->num_sms / base;
+      want = want < 1 ? 1 : (want > tiles ? tiles : want);
+      prefix_tps = (tiles + want - 1) / want;
+      prefix_slices = (tiles + prefix_tps - 1) / prefix_tps;  // no slice is empty
+      p.k_start = shared_prefix_len;
+      p.split_base = prefix_slices;
+    }
+    const int suffix_ctx = b->max_ctx_len - p.k_start;  // longest key range the streaming kernel covers, minus one
+    p.split_len = plan_split_len(h, b->batch, suffix_ctx);
+    p.grid_splits = plan_max_splits(p.split_len, suffix_ctx);
+    p.max_splits = p.split_base + p.grid_splits;
+    if (p.grid_splits > 65535) return HSWA_ERR_UNSUPPORTED;
     if (p.max_splits > 1) {
       const size_t rows = (size_t)b->batch * h->cfg.num_q_heads;
       const size_t o_bytes = (rows * p.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
@@ -274,7 +296,25 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
   // arrays) may start early: those kernels never write the batch arrays or another layer's pool.
   const bool early = h->chain_ok && k_new != nullptr && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len;
   h->chain_ok = 0;
-  if (hswa_launch_decode(h, tm, p, early, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (cascade) {
+    PrefillParams pp = {};
+    pp.m = p.m;
+    pp.b = p.b;
+    pp.pool = p.pool;
+    pp.num_pages = p.num_pages;
+    pp.is_swa = 0;
+    pp.q = p.q;
+    pp.err = h->err;
+    pp.prefix_len = shared_prefix_len;
+    pp.prefix_tiles_per_split = prefix_tps;
+    pp.max_splits = p.max_splits;
+    pp.part_o = p.part_o;
+    pp.part_ml = p.part_ml;
+    CUtensorMap tq;
+    if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->batch, 16, &tq, 8)) != HSWA_OK) return st;
+    if (hswa_launch_decode_prefix(tm, tq, pp, prefix_slices, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  }
+  if (hswa_launch_decode(h, tm, p, early && !cascade, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (k_new != nullptr) {
     h->chain_ok = 1;
@@ -282,6 +322,20 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
     h->chain_ctx = (const void*)b->ctx_len;
   }
   return HSWA_OK;
+}
+
+hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,
+                             const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  return decode_impl(h, layer, b, 0, q, k_new, v_new, out, lse, workspace, workspace_bytes, stream);
+}
+
+hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b,
+                                           int32_t shared_prefix_len, const void* q, const void* k_new, const void* v_new,
+                                           void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!h || shared_prefix_len < 0 || shared_prefix_len % h->cfg.page_size != 0) return HSWA_ERR_INVALID_ARG;
+  if (b && shared_prefix_len > b->max_ctx_len) return HSWA_ERR_INVALID_ARG;
+  return decode_impl(h, layer, b, shared_prefix_len, q, k_new, v_new, out, lse, workspace, workspace_bytes, stream);
 }
 
 hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* q,

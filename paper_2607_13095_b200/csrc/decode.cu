@@ -73,7 +73,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
   kr.head = 0;
   int k_begin = 0;
   if (!p.is_swa) {
-    k_begin = split * p.split_len;
+    k_begin = p.k_start + split * p.split_len;
     if (k_begin >= kv_len) return;
     kr.span = min(kv_len, k_begin + p.split_len) - k_begin;
   } else {
@@ -380,8 +380,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
         reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(val);
       if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
     } else {
-      p.part_o[(row * p.max_splits + split) * D + d] = O;
-      if (d == 0) p.part_ml[row * p.max_splits + split] = make_float2(mm, L);
+      p.part_o[(row * p.max_splits + p.split_base + split) * D + d] = O;
+      if (d == 0) p.part_ml[row * p.max_splits + p.split_base + split] = make_float2(mm, L);
     }
   }
 }
@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
   const int r = warp_global / M.Hq;
   const int64_t row = warp_global;
   const int kv_len = p.b.ctx_len[r] + 1;
-  const int n_splits = min(p.max_splits, (kv_len + p.split_len - 1) / p.split_len);
+  const int n_splits = min(p.max_splits, p.split_base + (kv_len - p.k_start + p.split_len - 1) / p.split_len);
   const float2* ml = p.part_ml + row * p.max_splits;
   const float* po = p.part_o + row * p.max_splits * D;
   float mm = -INFINITY;
@@ -448,7 +448,7 @@ cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool e
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.b.B, p.max_splits, p.m.Hkv);
+  cfg.gridDim = dim3(p.b.B, p.grid_splits, p.m.Hkv);
   cfg.blockDim = dim3((NW + 1) * 32, 1, 1);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = s;

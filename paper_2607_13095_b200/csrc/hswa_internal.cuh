@@ -59,7 +59,10 @@ struct DecodeParams {
   void* out;   // [B][Hq][D]
   float* lse;  // [B][Hq] or null
   int32_t split_len;   // keys per split (multiple of 64)
-  int32_t max_splits;  // grid extent; 1 = write final output directly
+  int32_t max_splits;  // partial slots per row; 1 = write final output directly
+  int32_t k_start;     // first key position this launch covers (cascade decode: the shared prefix length), else 0
+  int32_t split_base;  // partial slot of this launch's split 0
+  int32_t grid_splits; // splits this launch covers (grid extent)
   float* part_o;       // [B*Hq][max_splits][D]
   float2* part_ml;     // [B*Hq][max_splits] (m in log2 units, l)
   int32_t* err;
@@ -91,6 +94,12 @@ struct PrefillParams {
   int32_t total_q;
   int32_t max_q_len;
   int32_t* err;
+  // shared-prefix stage of cascade decode only
+  int32_t prefix_len;              // shared tokens (multiple of the page size)
+  int32_t prefix_tiles_per_split;  // 128-key tiles per prefix slice
+  int32_t max_splits;              // partial slots per (request, head) row
+  float* part_o;
+  float2* part_ml;
 };
 
 // Launchers implemented in the kernel translation units.
@@ -103,6 +112,8 @@ bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                    const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s);
 void hswa_prefill_packed_geometry(int G, int* tq, int* nkeys);
+cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const PrefillParams& p, int n_slices,
+                                      cudaStream_t s);
 cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                          const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int first_block,
                                          cudaStream_t s);

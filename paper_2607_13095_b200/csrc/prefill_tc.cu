@@ -165,6 +165,11 @@ __device__ __forceinline__ TileSeq tile_seq(int is_swa, int ctx, int b, int W, i
   return s;
 }
 
+// PREFIX = true turns the same pipeline into the shared-prefix stage of batched decode (paper Sec. 3.1.3 /
+// 3.1.4: requests that share a system prompt share its pages): the 128 rows of a Q tile are 16 requests x
+// the 8 query heads of one KV head, the keys are a slice of the shared prefix pages, nothing is masked, and
+// the block writes an unnormalised (m, l, o) partial per row for the split-K combine instead of an output.
+template <bool PREFIX>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_constant__ CUtensorMap tm_q,
                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -179,16 +184,37 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int pair = blockIdx.x, kh = blockIdx.y;
-  const int r = blockIdx.z % p.b.B;
-  const int b = max_tiles - 1 - (int)(blockIdx.z / p.b.B);  // longest tiles are scheduled first
-  const int t0 = p.b.q_indptr[r];
-  const int n = p.b.q_indptr[r + 1] - t0;
-  if (b * BM >= n) return;  // uniform for the block
+  int r, b, t0, n, ctx, head, h0, page_off = 0;
+  TileSeq seq;
+  if constexpr (PREFIX) {
+    // blockIdx.x = slice of the prefix, blockIdx.z = group of 32 requests (16 per Q tile)
+    r = blockIdx.z * 32;
+    if (r >= p.b.B) return;
+    b = 0;
+    t0 = r;
+    n = p.b.B - r;  // requests left from r on
+    head = 0;
+    h0 = kh * M.G;
+    const int tiles_total = (p.prefix_len + BN - 1) / BN;
+    const int tile_begin = blockIdx.x * p.prefix_tiles_per_split;
+    seq.nA = min(p.prefix_tiles_per_split, tiles_total - tile_begin);
+    seq.c_lo = 0;
+    seq.nB = 0;
+    page_off = 2 * tile_begin;
+    ctx = p.prefix_len - tile_begin * BN;  // keys from this slice's first tile to the end of the prefix
+    if (seq.nA <= 0) return;               // the host plans slices so that none is empty
+  } else {
+    r = blockIdx.z % p.b.B;
+    b = max_tiles - 1 - (int)(blockIdx.z / p.b.B);  // longest tiles are scheduled first
+    t0 = p.b.q_indptr[r];
+    n = p.b.q_indptr[r + 1] - t0;
+    if (b * BM >= n) return;  // uniform for the block
+    ctx = p.b.ctx_len[r];
+    head = p.is_swa ? p.b.ring_head[r] : 0;
+    h0 = kh * M.G + pair * 2;
+    seq = tile_seq(p.is_swa, ctx, b, M.W, M.R);
+  }
   if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;  // an earlier block gave up: do not queue behind it
-  const int ctx = p.b.ctx_len[r];
-  const int head = p.is_swa ? p.b.ring_head[r] : 0;
-  const int h0 = kh * M.G + pair * 2;
-  const TileSeq seq = tile_seq(p.is_swa, ctx, b, M.W, M.R);
   const int n_tiles = seq.total();
 
   auto bar = [&](int i) { return smem_u32(&bars[i]); };
@@ -228,11 +254,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       tma_prefetch_desc(&tm_v);
       mbar_arrive_expect_tx(bar(BAR_Q), 2 * TILE_BYTES);
       for (int i = 0; i < 2; ++i)
-        for (int hf = 0; hf < 2; ++hf)
-          tma_load_3d(sbase + OFF_Q + i * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(BAR_Q), hf * 64, h0 + i, t0 + b * BM);
+        for (int hf = 0; hf < 2; ++hf) {
+          if constexpr (PREFIX)  // box {64, 8 heads, 16 requests} over q [B][Hq][D]
+            tma_load_3d(sbase + OFF_Q + i * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(BAR_Q), hf * 64, h0, r + 16 * i);
+          else
+            tma_load_3d(sbase + OFF_Q + i * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(BAR_Q), hf * 64, h0 + i, t0 + b * BM);
+        }
     }
     // page ids of the cached tiles, 32 at a time
-    const int32_t* tbl = p.is_swa ? p.b.ring_table + (int64_t)r * M.R : p.b.block_table + (int64_t)r * p.b.max_blocks;
+    const int32_t* tbl = p.is_swa ? p.b.ring_table + (int64_t)r * M.R : p.b.block_table + (int64_t)r * p.b.max_blocks + page_off;
     const int n_pages = p.is_swa ? M.R : (ctx + PG - 1) / PG;
     int pid_next = lane < n_pages ? tbl[lane] : 0;
     int pid_cur = 0;
@@ -506,6 +536,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     const float l_other = xch[0][i][half ^ 1][rr];
     ok = ok && !__any_sync(0xffffffffu, l_other != l_other);
     const float l_tot = l_run + l_other;
+    if constexpr (PREFIX) {
+      // partial for the split-K combine: row = (request, head), unnormalised o with its (m, l)
+      const int rq = r + 16 * i + (rr >> 3);
+      const bool row_ok = ok && rq < p.b.B;
+      const int64_t prow = ((int64_t)rq * M.Hq + kh * M.G + (rr & 7)) * p.max_splits + blockIdx.x;
+#pragma unroll 1
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t w[32];
+        tmem_ld32(tO + c2 * 32, w);
+        tc_wait_ld();
+        if (row_ok) {
+          float4* dst = reinterpret_cast<float4*>(p.part_o + prow * HD + half * 64 + c2 * 32);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            dst[k] = make_float4(__uint_as_float(w[4 * k]), __uint_as_float(w[4 * k + 1]), __uint_as_float(w[4 * k + 2]),
+                                 __uint_as_float(w[4 * k + 3]));
+        }
+      }
+      if (row_ok && half == 0) p.part_ml[prow] = make_float2(m_st, l_tot);
+    } else {
     const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
     const bool row_ok = ok && ri < n;
     const int64_t orow = ((int64_t)(t0 + ri) * M.Hq + (h0 + i));
@@ -538,6 +588,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
     if (row_ok && half == 0 && p.lse)
       p.lse[orow] = l_tot > 0.f ? (m_st + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+    }
   }
 
   // ---- teardown: everyone is done with TMEM before it is released ----
@@ -1131,11 +1182,24 @@ cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensor
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                    const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s) {
   if (p.b.B == 0 || p.total_q == 0 || p.max_q_len == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
   int max_tiles = (p.max_q_len + BM - 1) / BM;
   if (tile_limit > 0 && tile_limit < max_tiles) max_tiles = tile_limit;
   dim3 grid(p.m.G / 2, p.m.Hkv, (unsigned)(p.b.B * max_tiles));
-  prefill_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
+  prefill_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
+  return cudaGetLastError();
+}
+
+// Shared-prefix stage of cascade decode: grid (prefix slices, KV heads, groups of 32 requests).  tm_q is the
+// packed map (box {64, 8 heads, 16 requests}) over q [B][Hq][D]; p carries prefix_len, the slice plan and the
+// partial buffers.
+cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const PrefillParams& p,
+                                      int n_slices, cudaStream_t s) {
+  if (p.b.B == 0 || n_slices <= 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  dim3 grid(n_slices, p.m.Hkv, (p.b.B + 31) / 32);
+  prefill_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_pool, tm_pool, p, 1);
   return cudaGetLastError();
 }

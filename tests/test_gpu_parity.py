@@ -366,3 +366,62 @@ def test_prefill_tc_sweep(d, is_swa):
     assert err <= TOL and lerr <= TOL, (err, lerr)
     err, _ = run_prefill(sc, is_swa, fuse_append=False, out_dtype=torch.bfloat16)
     assert err <= 2 * TOL, err   # bf16 output: rows with 1-3 keys can carry half a bf16 ulp of a value near 4
+
+
+@pytest.mark.parametrize("W", [64, 96, 33])
+@pytest.mark.parametrize("G", [8, 4, 2])
+def test_prefill_tc_other_windows(W, G):
+    """Windows other than the paper's 128: the pipelined SWA kernel is bypassed and the packed / tile kernels
+    must apply the general window mask."""
+    d = dims(G, 128, 64, 1, W=W)
+    ctx = [0, 1, W - 1, W, 200, 64]
+    q_len = [300, 130, 257, 129, 1, 700]
+    sc = build_scenario(d, ctx, q_len, seed=41 + W)
+    err, lerr = run_prefill(sc, True)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+    err, lerr = run_decode(build_scenario(d, [0, 1, W - 1, W, 5 * W + 3], [1] * 5, seed=42 + W), True, True)
+    assert err <= TOL and lerr <= TOL, (err, lerr)
+
+
+def test_prefill_tc_long_context_and_many_requests():
+    d = dims(8, 128, 64, 1)
+    ctx = [20000, 0, 4097] + [int(x) for x in np.random.default_rng(7).integers(0, 700, 13)]
+    q_len = [300, 2049, 128] + [int(x) for x in np.random.default_rng(8).integers(0, 400, 13)]
+    sc = build_scenario(d, ctx, q_len, seed=43)
+    for is_swa in (False, True):
+        err, lerr = run_prefill(sc, is_swa)
+        assert err <= TOL and lerr <= TOL, (is_swa, err, lerr)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# cascade decode over a shared prefix
+@pytest.mark.parametrize("G,Hkv,B,prefix_pages", [(8, 2, 40, 37), (8, 1, 5, 2), (8, 2, 33, 64), (4, 2, 6, 8)])
+def test_decode_shared_prefix(G, Hkv, B, prefix_pages):
+    d = dims(G, 128, 64, Hkv)
+    prefix = 64 * prefix_pages
+    rng = np.random.default_rng(50 + B)
+    ctx = [prefix + int(x) for x in rng.integers(0, 700, B)]
+    ctx[0] = prefix          # a request whose whole context is the shared prefix
+    sc = build_scenario(d, ctx, [1] * B, seed=51, shared_prefix_tokens=prefix)
+    t = sc.tables
+    assert (t.block_table[:, :prefix_pages] == t.block_table[0, :prefix_pages]).all()
+    h = make_handle(d)
+    q, k_new, v_new = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    ws = workspace_for(h, t)
+    for is_swa in (False, True):
+        pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+        layer = hb.Layer(pool, is_swa)
+        out = torch.full((B, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+        lse = torch.full((B, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+        hb.hswa_decode_attn_shared_prefix(h, layer, dev_batch(t, True), prefix, q, k_new, v_new, out, lse, ws)
+        check_no_async_error(h)
+        ol = sc.layer(is_swa)
+        ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+        got = out.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
+        orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+        assert np.array_equal(to_host_bits(pool), ol.pool)
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn_shared_prefix(h, layer, dev_batch(t, True), 65, q, k_new, v_new, out, lse, ws)
+    assert e.value.status == hb.HSWA_ERR_INVALID_ARG
