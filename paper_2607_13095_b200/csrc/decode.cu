@@ -42,6 +42,106 @@ struct KeyRange {
   }
 };
 
+// One consumer warp's work on a staged 64-key tile: zero the V rows of invisible keys, S^T = K Q^T, online
+// softmax for the warp's (m, l, O^T) state, O^T += V^T P^T.  (vm0, vm1) is the 64-bit visibility mask of the tile.
+template <int D>
+__device__ __forceinline__ void consume_tile(uint8_t* sV, uint32_t aK, uint32_t aV, uint32_t vm0, uint32_t vm1, bool wrote,
+                                             const uint32_t (&qf)[D / 16][2], float scale_log2, float (&m_run)[2],
+                                             float (&l_run)[2], float (&o)[D / 16][4], int lane) {
+  constexpr int HALF_BYTES = TK * 128;
+  constexpr int CHUNKS = D / 8;
+  constexpr int KS = D / 16;
+  const int mi = lane >> 3, mr = lane & 7;
+  if ((vm0 & vm1) != 0xffffffffu) {
+    // zero the V rows of invisible keys so that 0 * (stale or non-finite) cannot reach the output
+    for (int idx = lane; idx < TK * CHUNKS; idx += 32) {
+      const int row = idx / CHUNKS, ch = idx % CHUNKS;
+      const bool v = ((row < 32 ? vm0 : vm1) >> (row & 31)) & 1u;
+      if (!v) *reinterpret_cast<uint4*>(sV + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = make_uint4(0, 0, 0, 0);
+    }
+    wrote = true;
+  }
+  if (wrote) {
+    fence_proxy_async_smem();
+    __syncwarp();
+  }
+
+  if ((vm0 | vm1) != 0u) {
+    // S^T = K Q^T for the 64 keys (four 16-key blocks)
+    float s[4][4];
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+      s[kb][0] = s[kb][1] = s[kb][2] = s[kb][3] = 0.f;
+      const int key = kb * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int chunk = 2 * ks + (mi >> 1);
+        uint32_t a0, a1, a2, a3;
+        ldmatrix_x4(aK + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+        mma_bf16_16816(s[kb], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
+      }
+    }
+    // mask, scale, tile maxima per head (this thread: heads qd and qd+1; keys lane/4 + 8j)
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+      const int keyA = kb * 16 + (lane >> 2), keyB = keyA + 8;
+      const bool vA = ((keyA < 32 ? vm0 : vm1) >> (keyA & 31)) & 1u;
+      const bool vB = ((keyB < 32 ? vm0 : vm1) >> (keyB & 31)) & 1u;
+      s[kb][0] = vA ? s[kb][0] * scale_log2 : -INFINITY;
+      s[kb][1] = vA ? s[kb][1] * scale_log2 : -INFINITY;
+      s[kb][2] = vB ? s[kb][2] * scale_log2 : -INFINITY;
+      s[kb][3] = vB ? s[kb][3] * scale_log2 : -INFINITY;
+      mx[0] = fmaxf(mx[0], fmaxf(s[kb][0], s[kb][2]));
+      mx[1] = fmaxf(mx[1], fmaxf(s[kb][1], s[kb][3]));
+    }
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sh));
+      mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sh));
+    }
+    float m_use[2], alpha[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float m_new = fmaxf(m_run[j], mx[j]);
+      m_use[j] = m_new == -INFINITY ? 0.f : m_new;
+      alpha[j] = fast_exp2(m_run[j] - m_use[j]);
+      m_run[j] = m_new;
+      l_run[j] *= alpha[j];
+    }
+#pragma unroll
+    for (int i = 0; i < KS; ++i) {
+      o[i][0] *= alpha[0];
+      o[i][1] *= alpha[1];
+      o[i][2] *= alpha[0];
+      o[i][3] *= alpha[1];
+    }
+    uint32_t pk[8];
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+      pk[2 * kb] = pack_bf16x2(fast_exp2(s[kb][0] - m_use[0]), fast_exp2(s[kb][1] - m_use[1]));
+      pk[2 * kb + 1] = pack_bf16x2(fast_exp2(s[kb][2] - m_use[0]), fast_exp2(s[kb][3] - m_use[1]));
+      const float2 f0 = unpack_bf16x2(pk[2 * kb]), f1 = unpack_bf16x2(pk[2 * kb + 1]);
+      l_run[0] += f0.x + f1.x;  // sum the values the tensor core will actually multiply
+      l_run[1] += f0.y + f1.y;
+    }
+    // O^T += V^T P^T
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+      const uint32_t b0 = movmatrix_trans(pk[2 * kb]);
+      const uint32_t b1 = movmatrix_trans(pk[2 * kb + 1]);
+      const int key = kb * 16 + (mi >> 1) * 8 + mr;
+#pragma unroll
+      for (int mt = 0; mt < KS; ++mt) {
+        const int chunk = 2 * mt + (mi & 1);
+        uint32_t a0, a1, a2, a3;
+        ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+        mma_bf16_16816(o[mt], a0, a1, a2, a3, b0, b1);
+      }
+    }
+  }
+}
+
 template <int D, int P, int NS, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, 2)
 decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
@@ -190,7 +290,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
         qf[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
       }
     }
-    const int mi = lane >> 3, mr = lane & 7;
     for (int t = cw; t < n_tiles; t += NW) {
       const int stage = t % NS;
       if (!mbar_wait(smem_u32(&bars[stage]), (t / NS) & 1)) {
@@ -233,94 +332,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
       // validity of the tile's 64 keys
       const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
       const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
-      if ((vm0 & vm1) != 0xffffffffu) {
-        // zero the V rows of invisible keys so that 0 * (stale or non-finite) cannot reach the output
-        for (int idx = lane; idx < TK * CHUNKS; idx += 32) {
-          const int row = idx / CHUNKS, ch = idx % CHUNKS;
-          const bool v = ((row < 32 ? vm0 : vm1) >> (row & 31)) & 1u;
-          if (!v) *reinterpret_cast<uint4*>(sV + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = make_uint4(0, 0, 0, 0);
-        }
-        wrote = true;
-      }
-      if (wrote) {
-        fence_proxy_async_smem();
-        __syncwarp();
-      }
-
-      if ((vm0 | vm1) != 0u) {
-        // S^T = K Q^T for the 64 keys (four 16-key blocks)
-        float s[4][4];
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          s[kb][0] = s[kb][1] = s[kb][2] = s[kb][3] = 0.f;
-          const int key = kb * 16 + (mi & 1) * 8 + mr;
-#pragma unroll
-          for (int ks = 0; ks < KS; ++ks) {
-            const int chunk = 2 * ks + (mi >> 1);
-            uint32_t a0, a1, a2, a3;
-            ldmatrix_x4(aK + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
-            mma_bf16_16816(s[kb], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
-          }
-        }
-        // mask, scale, tile maxima per head (this thread: heads qd and qd+1; keys lane/4 + 8j)
-        float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          const int keyA = kb * 16 + (lane >> 2), keyB = keyA + 8;
-          const bool vA = ((keyA < 32 ? vm0 : vm1) >> (keyA & 31)) & 1u;
-          const bool vB = ((keyB < 32 ? vm0 : vm1) >> (keyB & 31)) & 1u;
-          s[kb][0] = vA ? s[kb][0] * M.scale_log2 : -INFINITY;
-          s[kb][1] = vA ? s[kb][1] * M.scale_log2 : -INFINITY;
-          s[kb][2] = vB ? s[kb][2] * M.scale_log2 : -INFINITY;
-          s[kb][3] = vB ? s[kb][3] * M.scale_log2 : -INFINITY;
-          mx[0] = fmaxf(mx[0], fmaxf(s[kb][0], s[kb][2]));
-          mx[1] = fmaxf(mx[1], fmaxf(s[kb][1], s[kb][3]));
-        }
-#pragma unroll
-        for (int sh = 4; sh <= 16; sh <<= 1) {
-          mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sh));
-          mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sh));
-        }
-        float m_use[2], alpha[2];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const float m_new = fmaxf(m_run[j], mx[j]);
-          m_use[j] = m_new == -INFINITY ? 0.f : m_new;
-          alpha[j] = fast_exp2(m_run[j] - m_use[j]);
-          m_run[j] = m_new;
-          l_run[j] *= alpha[j];
-        }
-#pragma unroll
-        for (int i = 0; i < KS; ++i) {
-          o[i][0] *= alpha[0];
-          o[i][1] *= alpha[1];
-          o[i][2] *= alpha[0];
-          o[i][3] *= alpha[1];
-        }
-        uint32_t pk[8];
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          pk[2 * kb] = pack_bf16x2(fast_exp2(s[kb][0] - m_use[0]), fast_exp2(s[kb][1] - m_use[1]));
-          pk[2 * kb + 1] = pack_bf16x2(fast_exp2(s[kb][2] - m_use[0]), fast_exp2(s[kb][3] - m_use[1]));
-          const float2 f0 = unpack_bf16x2(pk[2 * kb]), f1 = unpack_bf16x2(pk[2 * kb + 1]);
-          l_run[0] += f0.x + f1.x;  // sum the values the tensor core will actually multiply
-          l_run[1] += f0.y + f1.y;
-        }
-        // O^T += V^T P^T
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-          const uint32_t b0 = movmatrix_trans(pk[2 * kb]);
-          const uint32_t b1 = movmatrix_trans(pk[2 * kb + 1]);
-          const int key = kb * 16 + (mi >> 1) * 8 + mr;
-#pragma unroll
-          for (int mt = 0; mt < KS; ++mt) {
-            const int chunk = 2 * mt + (mi & 1);
-            uint32_t a0, a1, a2, a3;
-            ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
-            mma_bf16_16816(o[mt], a0, a1, a2, a3, b0, b1);
-          }
-        }
-      }
+      consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
     }
@@ -439,6 +451,278 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
   if (lane == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// SWA layers: persistent variant.  A ring holds at most C slots per (request, KV head), i.e. a handful of
+// tiles, so a block per ring is all latency: table reads, one TMA round trip, a short compute, a merge.
+// Here a block walks many rings: the producer warp streams the tiles of ring after ring through the same
+// stage buffers (metadata of the next ring fetched one ring ahead), the consumer warps prefetch the next
+// ring's Q while they work, and every ring's warps merge through a small scratch area.  The loads of ring
+// k + 1 thus overlap the compute, merge and output of ring k.
+template <int D, int P>
+__global__ void __launch_bounds__(128, 2)
+decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p, const int n_items) {
+  constexpr int NS = 3, NW = 3;
+  constexpr int HALVES = D / 64;
+  constexpr int PPT = TK / P;
+  constexpr int HALF_BYTES = TK * 128;
+  constexpr int STAGE_BYTES = 2 * HALVES * HALF_BYTES;
+  constexpr int BOX_BYTES = P * 128;
+  constexpr int CHUNKS = D / 8;
+  constexpr int KS = D / 16;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * NS];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  float* sc_o = reinterpret_cast<float*>(smem + NS * STAGE_BYTES);  // [NW][8][D]
+  float* sc_ml = sc_o + NW * 8 * D;                                 // [NW][8][2]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const ModelParams& M = p.m;
+  const int n_tiles = (M.C + TK - 1) / TK;
+  const bool fuse = p.k_new != nullptr;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(smem_u32(&bars[i]), 1);
+      mbar_init(smem_u32(&bars[NS + i]), 1);
+    }
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_pool);
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    // ---------------- producer ----------------
+    int it = blockIdx.x;
+    int ctx_n = 0, head_n = 0, pid_n = 0;
+    if (it < n_items) {
+      const int r = it / M.Hkv;
+      ctx_n = p.b.ctx_len[r];
+      head_n = p.b.ring_head[r];
+      pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : 0;
+    }
+    bool ok = true;
+    for (int k = 0; it < n_items && ok; ++k, it += gridDim.x) {
+      const int r = it / M.Hkv, kh = it % M.Hkv;
+      KeyRange kr;
+      kr.is_swa = 1;
+      kr.span = M.C;
+      kr.head = head_n;
+      kr.ctx = ctx_n;
+      kr.W = M.W;
+      kr.C = M.C;
+      const int pid = pid_n;
+      const int nxt = it + gridDim.x;
+      if (nxt < n_items) {  // next ring's metadata, one ring ahead of its first TMA
+        const int rn = nxt / M.Hkv;
+        ctx_n = p.b.ctx_len[rn];
+        head_n = p.b.ring_head[rn];
+        pid_n = lane < M.R ? p.b.ring_table[(int64_t)rn * M.R + lane] : 0;
+      }
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int g = k * n_tiles + t, stage = g % NS;
+        if (g >= NS && !mbar_wait(smem_u32(&bars[NS + stage]), ((g / NS) - 1) & 1)) {
+          if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 3);
+          ok = false;
+          break;
+        }
+        uint32_t need = 0;
+        int pages[PPT];
+#pragma unroll
+        for (int i = 0; i < PPT; ++i) {
+          const int pgi = t * PPT + i;
+          pages[i] = __shfl_sync(0xffffffffu, pid, pgi & 31);
+          bool v = false;
+          if (pgi < M.R)
+            for (int s = lane; s < P; s += 32) v |= kr.valid(pgi * P + s);
+          if (__any_sync(0xffffffffu, v)) need |= 1u << i;
+        }
+        if (lane == 0) {
+          uint32_t okm = 0;
+#pragma unroll
+          for (int i = 0; i < PPT; ++i) {
+            if (!(need & (1u << i))) continue;
+            if (pages[i] < 0 || pages[i] >= p.num_pages) {
+              record_error(p.err, HSWA_ERR_BOUNDS, r, t * PPT + i, pages[i]);
+              continue;
+            }
+            okm |= 1u << i;
+          }
+          const uint32_t full_bar = smem_u32(&bars[stage]);
+          if (okm == 0) {
+            mbar_arrive(full_bar);
+          } else {
+            mbar_arrive_expect_tx(full_bar, __popc(okm) * 2 * HALVES * BOX_BYTES);
+            const uint32_t sb = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+            for (int i = 0; i < PPT; ++i) {
+              if (!(okm & (1u << i))) continue;
+#pragma unroll
+              for (int kv = 0; kv < 2; ++kv)
+#pragma unroll
+                for (int hf = 0; hf < HALVES; ++hf)
+                  tma_load_4d(sb + (kv * HALVES + hf) * HALF_BYTES + i * BOX_BYTES, &tm_pool, full_bar, hf * 64, 0,
+                              kv * M.Hkv + kh, pages[i]);
+            }
+          }
+        }
+        __syncwarp();
+      }
+    }
+  } else {
+    // ---------------- consumers ----------------
+    const int cw = warp - 1;
+    const int g_row = lane >> 2;
+    const int qd = (lane & 3) * 2;
+    griddep_wait();  // q, k_new, v_new and out may belong to the previous kernel on the stream
+    griddep_launch_dependents();
+    int it = blockIdx.x;
+    uint32_t qn[KS][2];
+    int ctx_n = 0, head_n = 0;
+    auto prefetch = [&](int item) {
+      const int r = item / M.Hkv, kh = item % M.Hkv;
+      ctx_n = p.b.ctx_len[r];
+      head_n = p.b.ring_head[r];
+      const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qn[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+        qn[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+      }
+    };
+    if (it < n_items) prefetch(it);
+    for (int k = 0; it < n_items; ++k, it += gridDim.x) {
+      const int r = it / M.Hkv, kh = it % M.Hkv;
+      uint32_t qf[KS][2];
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qf[ks][0] = qn[ks][0];
+        qf[ks][1] = qn[ks][1];
+      }
+      KeyRange kr;
+      kr.is_swa = 1;
+      kr.span = M.C;
+      kr.head = head_n;
+      kr.ctx = ctx_n;
+      kr.W = M.W;
+      kr.C = M.C;
+      const int ctx = ctx_n;
+      if (it + gridDim.x < n_items) prefetch(it + gridDim.x);
+
+      float m_run[2] = {-INFINITY, -INFINITY};
+      float l_run[2] = {0.f, 0.f};
+      float o[KS][4];
+#pragma unroll
+      for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+      bool ok = true;
+      for (int t = cw; t < n_tiles; t += NW) {
+        const int g = k * n_tiles + t, stage = g % NS;
+        if (!mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {
+          if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
+          ok = false;
+          break;
+        }
+        uint8_t* sK = smem + stage * STAGE_BYTES;
+        uint8_t* sV = sK + HALVES * HALF_BYTES;
+        const uint32_t aK = smem_base + stage * STAGE_BYTES;
+        const uint32_t aV = aK + HALVES * HALF_BYTES;
+        const int tile_lo = t * TK;
+        bool wrote = false;
+        if (fuse && kr.head >= tile_lo && kr.head < tile_lo + TK) {
+          // fused append: the new token goes to ring slot ring_head, in the staged tile and in the cache
+          const int row = kr.head - tile_lo;
+          const int page = p.b.ring_table[(int64_t)r * M.R + kr.head / P];
+          const int slot = kr.head % P;
+          const bool page_ok = page >= 0 && page < p.num_pages;
+          if (!page_ok && lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, page);
+          for (int c = lane; c < 2 * CHUNKS; c += 32) {
+            const int kv = c / CHUNKS, ch = c % CHUNKS;
+            const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D + ch * 8;
+            const uint4 val = *reinterpret_cast<const uint4*>(src);
+            *reinterpret_cast<uint4*>((kv == 0 ? sK : sV) + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = val;
+            if (page_ok)
+              *reinterpret_cast<uint4*>(p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * P + slot) * D + ch * 8) = val;
+          }
+          wrote = true;
+        }
+        const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
+        const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
+        consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+      }
+      (void)ok;
+      (void)ctx;
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+      }
+      // merge the three warps' states through the scratch area and write the ring's output
+#pragma unroll
+      for (int mt = 0; mt < KS; ++mt) {
+        const int d0 = mt * 16 + (lane >> 2);
+        sc_o[(cw * 8 + qd) * D + d0] = o[mt][0];
+        sc_o[(cw * 8 + qd + 1) * D + d0] = o[mt][1];
+        sc_o[(cw * 8 + qd) * D + d0 + 8] = o[mt][2];
+        sc_o[(cw * 8 + qd + 1) * D + d0 + 8] = o[mt][3];
+      }
+      if (lane < 4) {
+        sc_ml[(cw * 8 + qd) * 2 + 0] = m_run[0];
+        sc_ml[(cw * 8 + qd) * 2 + 1] = l_run[0];
+        sc_ml[(cw * 8 + qd + 1) * 2 + 0] = m_run[1];
+        sc_ml[(cw * 8 + qd + 1) * 2 + 1] = l_run[1];
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
+      for (int idx = threadIdx.x - 32; idx < M.G * D; idx += NW * 32) {
+        const int g = idx / D, d = idx % D;
+        float mm = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sc_ml[(w * 8 + g) * 2]);
+        float L = 0.f, O = 0.f;
+        if (mm != -INFINITY) {
+#pragma unroll
+          for (int w = 0; w < NW; ++w) {
+            const float f = fast_exp2(sc_ml[(w * 8 + g) * 2] - mm);
+            L += f * sc_ml[(w * 8 + g) * 2 + 1];
+            O += f * sc_o[(w * 8 + g) * D + d];
+          }
+        }
+        const int64_t row = (int64_t)r * M.Hq + kh * M.G + g;
+        const float val = L > 0.f ? O / L : 0.f;
+        if (M.out_fp32)
+          reinterpret_cast<float*>(p.out)[row * D + d] = val;
+        else
+          reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(val);
+        if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");  // scratch may be rewritten
+    }
+  }
+}
+
+template <int D, int P>
+cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
+  constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
+  constexpr int SMEM = 3 * STAGE_BYTES + 3 * 8 * D * 4 + 3 * 8 * 2 * 4 + 1024;
+  auto kern = decode_ring_kernel<D, P>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  const int n_items = p.b.B * p.m.Hkv;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_items < 2 * h->num_sms ? n_items : 2 * h->num_sms, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, tm, p, n_items);
+}
+
 template <int D, int P, int NS, int NW>
 cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
@@ -462,10 +746,19 @@ cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool e
 
 }  // namespace
 
-cudaError_t hswa_launch_decode(const hswa_handle*, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
+cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
                                cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
   const int D = p.m.D, P = p.m.P;
+  if (p.is_swa) {  // rings: persistent blocks
+    if (D == 128 && P == 64) return launch_ring_t<128, 64>(h, tm_pool, p, early_start, s);
+    if (D == 128 && P == 32) return launch_ring_t<128, 32>(h, tm_pool, p, early_start, s);
+    if (D == 128 && P == 16) return launch_ring_t<128, 16>(h, tm_pool, p, early_start, s);
+    if (D == 64 && P == 64) return launch_ring_t<64, 64>(h, tm_pool, p, early_start, s);
+    if (D == 64 && P == 32) return launch_ring_t<64, 32>(h, tm_pool, p, early_start, s);
+    if (D == 64 && P == 16) return launch_ring_t<64, 16>(h, tm_pool, p, early_start, s);
+    return cudaErrorInvalidValue;
+  }
   if (D == 128 && P == 64) return launch_decode_t<128, 64, 3, 3>(tm_pool, p, early_start, s);
   if (D == 128 && P == 32) return launch_decode_t<128, 32, 3, 3>(tm_pool, p, early_start, s);
   if (D == 128 && P == 16) return launch_decode_t<128, 16, 3, 3>(tm_pool, p, early_start, s);
