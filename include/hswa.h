@@ -148,6 +148,19 @@ hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* lay
                                            const void* v_new, void* out, float* lse, void* workspace,
                                            size_t workspace_bytes, void* stream);
 
+/* Multi-token decode (paper Sec. 6.2: the models draft with 3 MTP layers, so a decode step verifies the last
+ * accepted token plus up to 3 drafts).  Every request has exactly q_len new tokens, 1 <= q_len <= 4;
+ * batch->q_indptr must be NULL, batch->total_q = B and batch->max_q_len = 1 as for hswa_decode_attn.
+ * q: device bf16 [B][q_len][Hq][D]; k_new, v_new: device bf16 [B][q_len][Hkv][D] (required); out: device
+ * [B][q_len][Hq][D]; lse: device fp32 [B][q_len][Hq] or NULL.  Token i of request r has position ctx[r] + i
+ * and attends causally (to the cache and to new tokens 0..i; on SWA layers inside its own window).  The q_len
+ * tokens are appended first (on a ring that is exact for q_len <= C - W + 1, checked), then one kernel streams
+ * the KV once for all q_len tokens.  Workspace: as hswa_decode_attn with max_total_q = max_batch * q_len.
+ * After the step call hswa_step_advance with a q_indptr describing the ACCEPTED tokens per request. */
+hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, int32_t q_len,
+                                 const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart of this
  * call; it exists for deployment reasons only.)
  * Same arguments, results and errors as hswa_decode_attn, minus the workspace: the split-K partials go to a

@@ -24,7 +24,7 @@ HSWA_ERR_TIMEOUT = 6
 
 EXPORTS = [
     "hswa_create", "hswa_destroy", "hswa_workspace_bytes", "hswa_validate_batch", "hswa_kv_append",
-    "hswa_decode_attn", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
+    "hswa_decode_attn", "hswa_decode_attn_mtp", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
 ]
 
 
@@ -83,6 +83,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_kv_append.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp]
     lib.hswa_decode_attn.restype = C.c_int
     lib.hswa_decode_attn.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.hswa_decode_attn_mtp.restype = C.c_int
+    lib.hswa_decode_attn_mtp.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), i32, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.hswa_decode_attn_shared_prefix.restype = C.c_int
     lib.hswa_decode_attn_shared_prefix.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), i32, vp, vp, vp, vp, vp,
                                                    vp, sz, vp]
@@ -195,6 +197,14 @@ def hswa_decode_attn(h: Handle, layer: Layer, batch: Batch, q, k_new, v_new, out
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().hswa_decode_attn(h.ptr, C.byref(layer.c), C.byref(batch.c), _ptr(q), _ptr(k_new), _ptr(v_new),
                                    _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes, _stream()), "hswa_decode_attn")
+
+
+def hswa_decode_attn_mtp(h: Handle, layer: Layer, batch: Batch, q_len: int, q, k_new, v_new, out, lse=None, workspace=None):
+    """Multi-token decode: q [B][q_len][Hq][D], k_new / v_new [B][q_len][Hkv][D], causal within the q_len drafts."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().hswa_decode_attn_mtp(h.ptr, C.byref(layer.c), C.byref(batch.c), int(q_len), _ptr(q), _ptr(k_new),
+                                       _ptr(v_new), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes, _stream()),
+           "hswa_decode_attn_mtp")
 
 
 def hswa_decode_attn_shared_prefix(h: Handle, layer: Layer, batch: Batch, shared_prefix_len: int, q, k_new, v_new, out,

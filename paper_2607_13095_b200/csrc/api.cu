@@ -182,7 +182,8 @@ void hswa_destroy(hswa_handle* h) {
 
 size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max_total_q, int32_t max_ctx_len) {
   if (!h || max_batch <= 0 || max_ctx_len < 0) return 0;
-  (void)max_total_q;  // prefill needs no scratch
+  // multi-token decode has max_total_q = batch x q_len rows; prefill needs no scratch
+  if (max_total_q > max_batch && max_total_q <= 4 * max_batch) max_batch = max_total_q;
   // Upper bound of rows * splits over every batch <= max_batch and context <= max_ctx_len under
   // plan_split_len: at the longest split length a row has ceil(kv / 2048) splits; a shorter length is only
   // chosen while batch * Hkv * splits stays below twice the fill target.
@@ -224,6 +225,7 @@ hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_b
   p.v_new = static_cast<const __nv_bfloat16*>(v_new);
   p.total_q = b->total_q;
   p.max_q_len = b->max_q_len;
+  p.uniform_n = 0;
   return hswa_launch_append(p, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
@@ -254,6 +256,7 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
   p.part_ml = nullptr;
   p.k_start = 0;
   p.split_base = 0;
+  p.nq = 1;
   // Cascade decode: the shared prefix is attended once per group of requests on the tensor cores, the
   // per-request suffixes by the streaming kernel; both leave partials for the combine.
   const bool cascade = !layer->is_swa && shared_prefix_len >= 128 && h->cfg.head_dim == 128 && h->cfg.page_size == 64 &&
@@ -328,6 +331,75 @@ hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa
                              const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, void* stream) {
   return decode_impl(h, layer, b, 0, q, k_new, v_new, out, lse, workspace, workspace_bytes, stream);
+}
+
+hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, int32_t q_len, const void* q,
+                                 const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  if (q_len == 1) return decode_impl(h, layer, b, 0, q, k_new, v_new, out, lse, workspace, workspace_bytes, stream);
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  h->chain_ok = 0;
+  if (b->q_indptr != nullptr || q_len < 1 || q_len > 4) return HSWA_ERR_INVALID_ARG;
+  if (b->batch == 0) return HSWA_OK;
+  if (!q || !out || !k_new || !v_new) return HSWA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return HSWA_ERR_INVALID_ARG;
+  if (layer->is_swa && q_len > h->ring_slots - h->cfg.window + 1) return HSWA_ERR_INVALID_ARG;  // append-then-attend limit
+
+  AppendParams a;
+  a.m = model_params(h);
+  a.b = batch_params(b);
+  a.pool = static_cast<__nv_bfloat16*>(layer->pool);
+  a.num_pages = layer->num_pages;
+  a.is_swa = layer->is_swa;
+  a.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  a.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  a.total_q = b->batch * q_len;
+  a.max_q_len = q_len;
+  a.uniform_n = q_len;
+
+  DecodeParams p;
+  p.m = a.m;
+  p.b = a.b;
+  p.pool = a.pool;
+  p.num_pages = a.num_pages;
+  p.is_swa = layer->is_swa;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = nullptr;  // the tokens are in the cache by the time the attention kernel runs
+  p.v_new = nullptr;
+  p.out = out;
+  p.lse = lse;
+  p.err = h->err;
+  p.part_o = nullptr;
+  p.part_ml = nullptr;
+  p.k_start = 0;
+  p.split_base = 0;
+  p.nq = q_len;
+  if (layer->is_swa) {
+    p.split_len = ((h->ring_slots + 63) / 64) * 64;
+    p.grid_splits = 1;
+  } else {
+    const int last = b->max_ctx_len + q_len - 1;  // highest key position
+    p.split_len = plan_split_len(h, b->batch, last);
+    p.grid_splits = plan_max_splits(p.split_len, last);
+    if (p.grid_splits > 65535) return HSWA_ERR_UNSUPPORTED;
+  }
+  p.max_splits = p.grid_splits;
+  if (p.max_splits > 1) {
+    const size_t rows = (size_t)b->batch * q_len * h->cfg.num_q_heads;
+    const size_t o_bytes = (rows * p.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
+    const size_t ml_bytes = (rows * p.max_splits * sizeof(float2) + 255) & ~size_t(255);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < o_bytes + ml_bytes)
+      return HSWA_ERR_WORKSPACE;
+    p.part_o = static_cast<float*>(workspace);
+    p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + o_bytes);
+  }
+  CUtensorMap tm;
+  if ((st = make_pool_map(h, layer, &tm)) != HSWA_OK) return st;
+  if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (hswa_launch_decode_mtp(tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  return HSWA_OK;
 }
 
 hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b,
@@ -411,6 +483,7 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
     a.v_new = p.v_new;
     a.total_q = p.total_q;
     a.max_q_len = p.max_q_len;
+    a.uniform_n = 0;
     if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   }
   return HSWA_OK;

@@ -31,8 +31,8 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
   const int kh = c / chunks_per_row;
   const int ch = c % chunks_per_row;
 
-  const int r = find_request(p.b, t);
-  const int t0 = p.b.q_indptr ? p.b.q_indptr[r] : r;
+  const int r = p.uniform_n > 0 ? t / p.uniform_n : find_request(p.b, t);
+  const int t0 = p.uniform_n > 0 ? r * p.uniform_n : (p.b.q_indptr ? p.b.q_indptr[r] : r);
   const int pos = p.b.ctx_len[r] + (t - t0);
   const int blk = pos / M.P;
   if (blk >= p.b.max_blocks) return;
@@ -51,8 +51,8 @@ __global__ void __launch_bounds__(256) append_ring_kernel(const AppendParams p) 
   const int chunks_per_row = M.D / 8;
   const int chunks_per_tok = 2 * M.Hkv * chunks_per_row;
   const int r = blockIdx.y;
-  const int t0 = p.b.q_indptr ? p.b.q_indptr[r] : r;
-  const int n = p.b.q_indptr ? p.b.q_indptr[r + 1] - t0 : 1;
+  const int t0 = p.uniform_n > 0 ? r * p.uniform_n : (p.b.q_indptr ? p.b.q_indptr[r] : r);
+  const int n = p.uniform_n > 0 ? p.uniform_n : (p.b.q_indptr ? p.b.q_indptr[r + 1] - t0 : 1);
   const int keep = min(n, M.C);
   const int gid = blockIdx.x * blockDim.x + threadIdx.x;
   if (gid >= keep * chunks_per_tok) return;

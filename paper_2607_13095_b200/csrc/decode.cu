@@ -43,20 +43,21 @@ struct KeyRange {
 };
 
 // One consumer warp's work on a staged 64-key tile: zero the V rows of invisible keys, S^T = K Q^T, online
-// softmax for the warp's (m, l, O^T) state, O^T += V^T P^T.  (vm0, vm1) is the 64-bit visibility mask of the tile.
+// softmax for the warp's (m, l, O^T) state, O^T += V^T P^T.  (vm0, vm1) is the 64-bit visibility mask of the tile for
+// this warp's query; V rows whose bit in (zm0, zm1) is clear are zeroed (rows no query of the block can see).
 template <int D>
 __device__ __forceinline__ void consume_tile(uint8_t* sV, uint32_t aK, uint32_t aV, uint32_t vm0, uint32_t vm1, bool wrote,
                                              const uint32_t (&qf)[D / 16][2], float scale_log2, float (&m_run)[2],
-                                             float (&l_run)[2], float (&o)[D / 16][4], int lane) {
+                                             float (&l_run)[2], float (&o)[D / 16][4], int lane, uint32_t zm0, uint32_t zm1) {
   constexpr int HALF_BYTES = TK * 128;
   constexpr int CHUNKS = D / 8;
   constexpr int KS = D / 16;
   const int mi = lane >> 3, mr = lane & 7;
-  if ((vm0 & vm1) != 0xffffffffu) {
+  if ((zm0 & zm1) != 0xffffffffu) {
     // zero the V rows of invisible keys so that 0 * (stale or non-finite) cannot reach the output
     for (int idx = lane; idx < TK * CHUNKS; idx += 32) {
       const int row = idx / CHUNKS, ch = idx % CHUNKS;
-      const bool v = ((row < 32 ? vm0 : vm1) >> (row & 31)) & 1u;
+      const bool v = ((row < 32 ? zm0 : zm1) >> (row & 31)) & 1u;
       if (!v) *reinterpret_cast<uint4*>(sV + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = make_uint4(0, 0, 0, 0);
     }
     wrote = true;
@@ -332,7 +333,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
       // validity of the tile's 64 keys
       const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
       const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
-      consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane);
+      consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
     }
@@ -405,10 +406,10 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
   const int lane = threadIdx.x & 31;
   const ModelParams& M = p.m;
   griddep_launch_dependents();  // the next attention kernel may start its cache loads now
-  if (warp_global >= p.b.B * M.Hq) return;
-  const int r = warp_global / M.Hq;
+  if (warp_global >= p.b.B * p.nq * M.Hq) return;
+  const int r = warp_global / (p.nq * M.Hq);
   const int64_t row = warp_global;
-  const int kv_len = p.b.ctx_len[r] + 1;
+  const int kv_len = p.b.ctx_len[r] + p.nq;
   const int n_splits = min(p.max_splits, p.split_base + (kv_len - p.k_start + p.split_len - 1) / p.split_len);
   const float2* ml = p.part_ml + row * p.max_splits;
   const float* po = p.part_o + row * p.max_splits * D;
@@ -648,7 +649,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         }
         const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
         const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
-        consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane);
+        consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
       }
@@ -723,6 +724,248 @@ cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const Dec
   return cudaLaunchKernelEx(&cfg, kern, tm, p, n_items);
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Multi-token decode (paper Sec. 6.2: the model drafts with 3 MTP layers, so a decode step carries the last
+// accepted token plus up to 3 drafts per request).  The nq new tokens are already in the cache (the append
+// runs first on the stream: on a ring that is safe for nq <= C - W + 1).  One consumer warp per draft token:
+// every warp walks every staged tile with its own Q, its own causal / window mask and its own softmax state,
+// so the KV bytes are streamed once for all nq tokens and no cross-warp merge is needed.
+struct KeyRangeMulti {
+  int is_swa, span, k_begin, head, ctx, W, C, nq;
+  __device__ __forceinline__ int slot_pos(int idx) const {  // position held by ring slot idx after the append
+    int off = idx - head;
+    if (off < 0) off += C;
+    return off < nq ? ctx + off : ctx + off - C;
+  }
+  // visible to draft token w (absolute position ctx + w)?
+  __device__ __forceinline__ bool valid(int idx, int w) const {
+    if (!is_swa) return idx < span && k_begin + idx <= ctx + w;
+    if (idx >= C) return false;
+    const int pos = slot_pos(idx);
+    return pos >= 0 && pos <= ctx + w && pos > ctx + w - W;
+  }
+  // visible to at least one of the nq tokens?
+  __device__ __forceinline__ bool any(int idx) const {
+    if (!is_swa) return idx < span;
+    if (idx >= C) return false;
+    const int pos = slot_pos(idx);
+    return pos >= 0 && pos <= ctx + nq - 1 && pos > ctx - W;
+  }
+};
+
+template <int D, int P, int NS>
+__global__ void __launch_bounds__(160, 2)
+decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
+  constexpr int HALVES = D / 64;
+  constexpr int PPT = TK / P;
+  constexpr int HALF_BYTES = TK * 128;
+  constexpr int STAGE_BYTES = 2 * HALVES * HALF_BYTES;
+  constexpr int BOX_BYTES = P * 128;
+  constexpr int KS = D / 16;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * NS];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+
+  const int r = blockIdx.x, split = blockIdx.y, kh = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const ModelParams& M = p.m;
+  const int nq = p.nq;
+  const int ctx = p.b.ctx_len[r];
+  const int kv_len = ctx + nq;
+
+  KeyRangeMulti kr;
+  kr.is_swa = p.is_swa;
+  kr.ctx = ctx;
+  kr.W = M.W;
+  kr.C = M.C;
+  kr.nq = nq;
+  kr.head = 0;
+  kr.k_begin = 0;
+  if (!p.is_swa) {
+    kr.k_begin = split * p.split_len;
+    if (kr.k_begin >= kv_len) return;
+    kr.span = min(kv_len, kr.k_begin + p.split_len) - kr.k_begin;
+  } else {
+    if (split > 0) return;
+    kr.head = p.b.ring_head[r];
+    kr.span = M.C;
+  }
+  const int n_tiles = (kr.span + TK - 1) / TK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(smem_u32(&bars[i]), 1);        // full: producer's arrive + TMA bytes
+      mbar_init(smem_u32(&bars[NS + i]), nq);  // empty: every consumer warp reads every tile
+    }
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_pool);
+  }
+  __syncthreads();
+
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+  float o[KS][4];
+#pragma unroll
+  for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  const int qd = (lane & 3) * 2;
+
+  if (warp == 0) {
+    const int32_t* tbl;
+    int n_pages;
+    if (!p.is_swa) {
+      tbl = p.b.block_table + (int64_t)r * p.b.max_blocks + kr.k_begin / P;
+      n_pages = (kr.span + P - 1) / P;
+    } else {
+      tbl = p.b.ring_table + (int64_t)r * M.R;
+      n_pages = M.R;
+    }
+    int pid_next = lane < n_pages ? tbl[lane] : 0;
+    int pid_cur = 0;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int pg0 = t * PPT;
+      if ((pg0 & 31) == 0) {
+        pid_cur = pid_next;
+        const int nx = pg0 + 32 + lane;
+        pid_next = nx < n_pages ? tbl[nx] : 0;
+      }
+      const int stage = t % NS;
+      if (t >= NS && !mbar_wait(smem_u32(&bars[NS + stage]), ((t / NS) - 1) & 1)) {
+        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 5);
+        break;
+      }
+      uint32_t need = 0;
+      int pages[PPT];
+#pragma unroll
+      for (int i = 0; i < PPT; ++i) {
+        const int pgi = pg0 + i;
+        pages[i] = __shfl_sync(0xffffffffu, pid_cur, pgi & 31);
+        bool v = false;
+        if (pgi < n_pages)
+          for (int s = lane; s < P; s += 32) v |= kr.any(pgi * P + s);
+        if (__any_sync(0xffffffffu, v)) need |= 1u << i;
+      }
+      if (lane == 0) {
+        uint32_t ok = 0;
+#pragma unroll
+        for (int i = 0; i < PPT; ++i) {
+          if (!(need & (1u << i))) continue;
+          if (pages[i] < 0 || pages[i] >= p.num_pages) {
+            record_error(p.err, HSWA_ERR_BOUNDS, r, pg0 + i, pages[i]);
+            continue;
+          }
+          ok |= 1u << i;
+        }
+        const uint32_t full_bar = smem_u32(&bars[stage]);
+        if (ok == 0) {
+          mbar_arrive(full_bar);
+        } else {
+          mbar_arrive_expect_tx(full_bar, __popc(ok) * 2 * HALVES * BOX_BYTES);
+          const uint32_t sb = smem_base + stage * STAGE_BYTES;
+#pragma unroll
+          for (int i = 0; i < PPT; ++i) {
+            if (!(ok & (1u << i))) continue;
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv)
+#pragma unroll
+              for (int hf = 0; hf < HALVES; ++hf)
+                tma_load_4d(sb + (kv * HALVES + hf) * HALF_BYTES + i * BOX_BYTES, &tm_pool, full_bar, hf * 64, 0,
+                            kv * M.Hkv + kh, pages[i]);
+          }
+        }
+      }
+      __syncwarp();
+    }
+  } else if (warp <= nq) {
+    const int w = warp - 1;  // draft token
+    const int g_row = lane >> 2;
+    uint32_t qf[KS][2];
+    {
+      const __nv_bfloat16* qrow = p.q + (((int64_t)r * nq + w) * M.Hq + kh * M.G + g_row) * D;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qf[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+        qf[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+      }
+    }
+    for (int t = 0; t < n_tiles; ++t) {
+      const int stage = t % NS;
+      if (!mbar_wait(smem_u32(&bars[stage]), (t / NS) & 1)) {
+        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 6);
+        break;
+      }
+      uint8_t* sV = smem + stage * STAGE_BYTES + HALVES * HALF_BYTES;
+      const uint32_t aK = smem_base + stage * STAGE_BYTES;
+      const uint32_t aV = aK + HALVES * HALF_BYTES;
+      const int tile_lo = t * TK;
+      const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane, w));
+      const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane, w));
+      const uint32_t zm0 = __ballot_sync(0xffffffffu, kr.any(tile_lo + lane));
+      const uint32_t zm1 = __ballot_sync(0xffffffffu, kr.any(tile_lo + 32 + lane));
+      consume_tile<D>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, zm0, zm1);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+    }
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+      l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+    }
+  }
+  __syncthreads();  // every tile has been consumed: the stage buffers now hold the per-token results
+  float* sc_o = reinterpret_cast<float*>(smem);  // [nq][8][D]
+  float* sc_ml = sc_o + 4 * 8 * D;               // [nq][8][2]
+  if (warp >= 1 && warp <= nq) {
+    const int w = warp - 1;
+#pragma unroll
+    for (int mt = 0; mt < KS; ++mt) {
+      const int d0 = mt * 16 + (lane >> 2);
+      sc_o[(w * 8 + qd) * D + d0] = o[mt][0];
+      sc_o[(w * 8 + qd + 1) * D + d0] = o[mt][1];
+      sc_o[(w * 8 + qd) * D + d0 + 8] = o[mt][2];
+      sc_o[(w * 8 + qd + 1) * D + d0 + 8] = o[mt][3];
+    }
+    if (lane < 4) {
+      sc_ml[(w * 8 + qd) * 2 + 0] = m_run[0];
+      sc_ml[(w * 8 + qd) * 2 + 1] = l_run[0];
+      sc_ml[(w * 8 + qd + 1) * 2 + 0] = m_run[1];
+      sc_ml[(w * 8 + qd + 1) * 2 + 1] = l_run[1];
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < nq * M.G * D; idx += blockDim.x) {
+    const int w = idx / (M.G * D), g = (idx / D) % M.G, d = idx % D;
+    const float mm = sc_ml[(w * 8 + g) * 2], L = sc_ml[(w * 8 + g) * 2 + 1], O = sc_o[(w * 8 + g) * D + d];
+    const int64_t row = ((int64_t)r * nq + w) * M.Hq + kh * M.G + g;
+    if (p.max_splits == 1) {
+      const float val = L > 0.f ? O / L : 0.f;
+      if (M.out_fp32)
+        reinterpret_cast<float*>(p.out)[row * D + d] = val;
+      else
+        reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(val);
+      if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    } else {
+      p.part_o[(row * p.max_splits + split) * D + d] = O;
+      if (d == 0) p.part_ml[row * p.max_splits + split] = make_float2(mm, L);
+    }
+  }
+}
+
+template <int D, int P, int NS>
+cudaError_t launch_mtp_t(const CUtensorMap& tm, const DecodeParams& p, cudaStream_t s) {
+  constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
+  constexpr int SMEM = NS * STAGE_BYTES + 1024;
+  static_assert(4 * 8 * D * 4 + 4 * 64 <= NS * STAGE_BYTES, "per-token results must fit the stage buffers");
+  auto kern = decode_mtp_kernel<D, P, NS>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (e != cudaSuccess) return e;
+  dim3 grid(p.b.B, p.grid_splits, p.m.Hkv);
+  kern<<<grid, (p.nq + 1) * 32, SMEM, s>>>(tm, p);
+  return cudaGetLastError();
+}
+
 template <int D, int P, int NS, int NW>
 cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
@@ -769,7 +1012,7 @@ cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool,
 }
 
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
-  const int rows = p.b.B * p.m.Hq;
+  const int rows = p.b.B * p.nq * p.m.Hq;
   if (rows == 0) return cudaSuccess;
   const int blocks = (rows * 32 + 127) / 128;
   if (p.m.D == 128)
@@ -777,4 +1020,17 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
   else
     combine_kernel<64><<<blocks, 128, 0, s>>>(p);
   return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_decode_mtp(const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
+  if (p.b.B == 0) return cudaSuccess;
+  if (p.nq < 1 || p.nq > 4) return cudaErrorInvalidValue;
+  const int D = p.m.D, P = p.m.P;
+  if (D == 128 && P == 64) return launch_mtp_t<128, 64, 3>(tm_pool, p, s);
+  if (D == 128 && P == 32) return launch_mtp_t<128, 32, 3>(tm_pool, p, s);
+  if (D == 128 && P == 16) return launch_mtp_t<128, 16, 3>(tm_pool, p, s);
+  if (D == 64 && P == 64) return launch_mtp_t<64, 64, 4>(tm_pool, p, s);
+  if (D == 64 && P == 32) return launch_mtp_t<64, 32, 4>(tm_pool, p, s);
+  if (D == 64 && P == 16) return launch_mtp_t<64, 16, 4>(tm_pool, p, s);
+  return cudaErrorInvalidValue;
 }

@@ -63,6 +63,7 @@ struct DecodeParams {
   int32_t k_start;     // first key position this launch covers (cascade decode: the shared prefix length), else 0
   int32_t split_base;  // partial slot of this launch's split 0
   int32_t grid_splits; // splits this launch covers (grid extent)
+  int32_t nq;          // new tokens per request (1; 2-4 for multi-token decode)
   float* part_o;       // [B*Hq][max_splits][D]
   float2* part_ml;     // [B*Hq][max_splits] (m in log2 units, l)
   int32_t* err;
@@ -78,6 +79,7 @@ struct AppendParams {
   const __nv_bfloat16* v_new;
   int32_t total_q;
   int32_t max_q_len;  // host-known bound of new tokens per request
+  int32_t uniform_n;  // > 0: every request has exactly this many new tokens and q_indptr is ignored
 };
 
 struct PrefillParams {
@@ -107,6 +109,7 @@ cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s);
 cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
                                cudaStream_t s);
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
+cudaError_t hswa_launch_decode_mtp(const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
 bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,

@@ -425,3 +425,33 @@ def test_decode_shared_prefix(G, Hkv, B, prefix_pages):
     with pytest.raises(hb.HswaError) as e:
         hb.hswa_decode_attn_shared_prefix(h, layer, dev_batch(t, True), 65, q, k_new, v_new, out, lse, ws)
     assert e.value.status == hb.HSWA_ERR_INVALID_ARG
+
+
+# ---------------------------------------------------------------------------------------------------------
+# multi-token (MTP) decode
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(4, 64, 16, 1), dims(3, 128, 32)], ids=str)
+@pytest.mark.parametrize("nq", [2, 4])
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_decode_mtp(d, nq, is_swa):
+    W, P, C = d.window, d.page_size, d.ring_slots
+    ctx = sorted({0, 1, 63, 64, W - 2, W - 1, W, W + 1, P - 1, P, C - 1, C, C + 1, 3 * C + 5, 2047, 2048, 2049, 5000})
+    B = len(ctx)
+    sc = build_scenario(d, ctx, [nq] * B, seed=60 + nq, ring_keep=C)
+    t = sc.tables
+    h = make_handle(d)
+    pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+    layer = hb.Layer(pool, is_swa)
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None, max_q_len=1,
+                 total_q=B, max_ctx_len=t.max_ctx_len)
+    out = torch.full((B * nq, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((B * nq, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(hb.hswa_workspace_bytes(h, B, B * nq, t.max_ctx_len + nq) + 256, dtype=torch.uint8, device="cuda")
+    hb.hswa_decode_attn_mtp(h, layer, b, nq, to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new), out, lse, ws)
+    check_no_async_error(h)
+    ol = sc.layer(is_swa)
+    ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)   # oracle: q_indptr with nq per request
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
+    orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+    assert np.array_equal(to_host_bits(pool), ol.pool)
