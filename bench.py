@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
+    ap.add_argument("--mtp", type=int, default=1, help="decode q_len per request (2-4: hswa_decode_attn_mtp)")
     ap.add_argument("--cascade", action="store_true", help="cfg4: use hswa_decode_attn_shared_prefix on the shared prefix")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill block reported under 'extra'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -132,15 +133,16 @@ class ClockSampler:
 class DecodeBench:
     """Device-resident state of a decode workload and one-step runner."""
 
-    def __init__(self, w, total_steps, device, cascade=False):
+    def __init__(self, w, total_steps, device, cascade=False, mtp=1):
         self.shared_prefix = w.tables.shared_prefix_pages * w.dims.page_size if cascade else 0
+        self.mtp = mtp
         import torch
         from paper_2607_13095_b200 import binding as hb
         from paper_2607_13095_b200 import workloads as wl
         self.torch, self.hb, self.w = torch, hb, w
         d, t0 = w.dims, w.tables
         # page ids for the contexts plus the tokens the run will append
-        self.t = wl.make_tables(d, t0.ctx_len, np.full(t0.batch, total_steps + 1), w.seed,
+        self.t = wl.make_tables(d, t0.ctx_len, np.full(t0.batch, total_steps + 1 + mtp), w.seed,
                                 shared_prefix_tokens=t0.shared_prefix_pages * d.page_size, slack=1.0)
         t = self.t
         g = torch.Generator(device=device)
@@ -153,7 +155,7 @@ class DecodeBench:
             pool = torch.empty((n_pages, 2, d.num_kv_heads, d.page_size, d.head_dim), dtype=torch.bfloat16, device=device)
             pool.normal_(generator=g)
             self.layers.append(hb.Layer(pool, is_swa))
-        L, B = len(self.layers), t.batch
+        L, B = len(self.layers), t.batch * mtp
         self.q = torch.randn((L, B, d.num_q_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
         self.k_new = torch.randn((L, B, d.num_kv_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
         self.v_new = torch.randn((L, B, d.num_kv_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
@@ -161,10 +163,11 @@ class DecodeBench:
         i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
         self.ctx0, self.head0 = i32(t.ctx_len), i32(t.ring_head)
         self.ctx, self.head = self.ctx0.clone(), self.head0.clone()
-        self.max_ctx = int(t.ctx_len.max()) + total_steps + 1
+        B = t.batch
+        self.max_ctx = int(t.ctx_len.max()) + total_steps + 1 + mtp
         self.batch = hb.Batch(self.ctx, i32(t.block_table), i32(t.ring_table), self.head, None, max_q_len=1,
                               total_q=B, max_ctx_len=self.max_ctx)
-        ws_bytes = hb.hswa_workspace_bytes(self.h, B, B, self.max_ctx)
+        ws_bytes = hb.hswa_workspace_bytes(self.h, B, B * mtp, self.max_ctx)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=device)
         self.full_idx = [i for i, s in enumerate(w.layer_is_swa) if not s]
         self.launches_per_step = sum(1 if s else (3 if self.shared_prefix else 2) for s in w.layer_is_swa) + 1
@@ -179,7 +182,10 @@ class DecodeBench:
             timed = events is not None and i == self.full_idx[0]
             if timed:
                 events[0].record()
-            if self.shared_prefix:
+            if self.mtp > 1:
+                hb.hswa_decode_attn_mtp(self.h, layer, self.batch, self.mtp, self.q[i], self.k_new[i], self.v_new[i],
+                                        self.out[i], None, self.ws)
+            elif self.shared_prefix:
                 hb.hswa_decode_attn_shared_prefix(self.h, layer, self.batch, self.shared_prefix, self.q[i], self.k_new[i],
                                                   self.v_new[i], self.out[i], None, self.ws)
             else:
@@ -448,7 +454,7 @@ def main():
         return
     w = make_workload(args.workload, seed_offset=rank, layers=args.layers, batch=args.batch)
     total_steps = args.steps + args.warmup
-    bench = DecodeBench(w, 2 * total_steps + 8, device, cascade=args.cascade)
+    bench = DecodeBench(w, 2 * total_steps + 8, device, cascade=args.cascade, mtp=args.mtp)
     t, d = bench.t, w.dims
 
     def barrier():
@@ -479,7 +485,7 @@ def main():
     if world > 1:
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
     ms_step = float(tmax.item()) / args.steps
-    tokens_per_step = t.batch * world
+    tokens_per_step = t.batch * world * args.mtp  # with --mtp: query tokens scored per step (1 accepted + drafts)
     value = tokens_per_step / (ms_step * 1e-3)
 
     # ---- end to end: pinned host inputs -> device, step, result -> host, every step ----
@@ -537,7 +543,7 @@ def main():
                    "batch": t.batch, "num_q_heads": d.num_q_heads, "num_kv_heads": d.num_kv_heads,
                    "head_dim": d.head_dim, "page_size": d.page_size, "window": d.window,
                    "ctx_sum": int(t.ctx_len.sum()), "shared_prefix_tokens": t.shared_prefix_pages * d.page_size,
-                   "cascade": bool(args.cascade), "l2": "inputs larger than L2 (Full-layer KV streamed per step "
+                   "cascade": bool(args.cascade), "mtp_q_len": args.mtp, "l2": "inputs larger than L2 (Full-layer KV streamed per step "
                    "exceeds 126 MB and evicts the SWA rings between reuses)", "out_dtype": "bf16"},
         "step_gbs": step_bytes / (ms_step * 1e-3) / 1e9 * world,
         "step_frac_of_measured_hbm": step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
