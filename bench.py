@@ -34,7 +34,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep"])
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
@@ -355,6 +355,36 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_prefix_sweep(args, torch, device, peaks):
+    """Paper Sec. 5.2 (figure: relative prefill throughput vs cached sequence length with a fixed 16K compute
+    chunk): one request, a 16 384-token chunk, cached prefix 0 / 64K / 256K / 1M tokens (the paper's length
+    buckets), attention of one hybrid block (1 Full + 6 SWA layers) only.  Prints tokens/s per prefix and the
+    throughput relative to the empty prefix."""
+    from paper_2607_13095_b200 import accounting
+    from paper_2607_13095_b200 import workloads as wl
+    chunk = args.chunk or 16384
+    rows = []
+    for prefix in (0, 65536, 262144, 1048576):
+        t = wl.make_tables(wl.BIG, [prefix], [chunk], seed=7, slack=1.0)
+        w = wl.Workload(f"prefix{prefix}-chunk{chunk}", wl.BIG, wl.hybrid_layer_flags(7)[:2], t, 7)
+        pb = PrefillBench(w, device)
+        ms_full = time_events(torch, lambda: pb.run_layer(0), 1, max(1, args.steps // 10))
+        ms_swa = time_events(torch, lambda: pb.run_layer(1), 2, 10)
+        block_ms = ms_full + 6 * ms_swa
+        rows.append({"prefix": prefix, "full_layer_ms": ms_full, "swa_layer_ms": ms_swa, "block_ms": block_ms,
+                     "tokens_per_s": chunk / (block_ms * 1e-3),
+                     "full_layer_tflops": accounting.prefill_flops(w, False) / (ms_full * 1e-3) / 1e12})
+        del pb
+        torch.cuda.empty_cache()
+    base = rows[0]["tokens_per_s"]
+    for r_ in rows:
+        r_["relative"] = r_["tokens_per_s"] / base
+    print(json.dumps({"metric": "prefill_attn_relative_throughput_vs_prefix", "unit": "x", "chunk": chunk,
+                      "value": rows[-1]["relative"], "rows": rows, "n_gpus": 1, "data": "synthetic", "dtype": "bf16",
+                      "note": "attention + append of one 1 Full + 6 SWA block; the paper's whole-model curve falls to "
+                              "about 0.12x at a 1M prefix (unnamed GPU), attention alone falls further"}))
+
+
 def run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks):
     """--workload cfg3: the chunked-prefill block as the measured workload (value = attention TFLOP/s of the
     whole 1 Full + 6 SWA block, fused append included)."""
@@ -449,6 +479,9 @@ def main():
     hb.load()
     peaks = measured_peaks()
 
+    if args.workload == "prefix_sweep":
+        run_prefix_sweep(args, torch, device, peaks)
+        return
     if args.workload == "cfg3":
         run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks)
         return
