@@ -34,7 +34,8 @@
  * torch scaled_dot_product_attention in fp64, SWA == Full while length <= W, ring == contiguous cache,
  * page-permutation invariance, shared-prefix equivalence, chunking invariance, closed forms (uniform
  * weights, constant V, single key, dominant logit), the paper's ~1/7 accounting ratio, ring storage law,
- * sequential-overwrite append exactness.  No function here is "parity unpinned".
+ * sequential-overwrite append exactness; window-safe length against a brute-force scan, window gather / scatter
+ * against the logical sequences, a round trip and an equivalent append.  No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -276,4 +277,78 @@ int64_t orc_attended_keys(const orc_config* cfg, int32_t is_swa, int64_t p) {
   int64_t full = p + 1;
   if (!is_swa) return full;
   return full < cfg->window ? full : (int64_t)cfg->window;
+}
+
+/* ---------------------------------------------------------------------------------------------------------
+ * SWA-aware prefix reuse (paper Sec. 3.1.3, "SWA-Aware Prefix Cache Tree", and Sec. 3.1.1 "Data movement").
+ *
+ * Window-safe length (item 1 of Sec. 3.1.3): a donor node matches the new request on its first match_len
+ * tokens; its Full KV is complete, but its SWA KV survives only where swa_valid[i] != 0.  A hit of length L is
+ * usable only if the tail of the hit that the next token's window needs still has valid SWA slots.  Reading
+ * taken (the paper says "the tail W tokens"; with the window including the query's own position the next
+ * token at position L needs exactly the W - 1 cached positions [L - W + 1, L)): L is safe iff every position
+ * in [max(0, L - (W - 1)), L) is valid.  Returns the largest safe L <= match_len (0 is always safe). */
+int64_t orc_window_safe_len(int64_t match_len, int32_t window, const uint8_t* swa_valid) {
+  for (int64_t L = match_len; L > 0; --L) {
+    int64_t lo = L - (window - 1);
+    if (lo < 0) lo = 0;
+    int ok = 1;
+    for (int64_t i = lo; i < L; ++i)
+      if (!swa_valid[i]) {
+        ok = 0;
+        break;
+      }
+    if (ok) return L;
+  }
+  return 0;
+}
+
+/* Window gather / scatter (Sec. 3.1.1: cross-tier transfers move only valid window data; Sec. 3.1.2: layerwise
+ * loadback).  The compact buffer holds, for request r, the W - 1 cached positions the next token's window needs:
+ * buf[((r * (W - 1) + j) * 2 + kv) * Hkv * D + h * D + d] for j = 0 .. W - 2, position ctx[r] - (W - 1) + j.
+ * Positions below 0 are zero in the buffer (gather) and skipped (scatter).  Gather reads the ring as it is;
+ * scatter writes the ring slots those positions map to under the batch's ring_head / ring_table. */
+int orc_window_gather(const orc_config* cfg, const orc_layer* L, const orc_batch* b, uint16_t* buf) {
+  const int Hkv = cfg->num_kv_heads, D = cfg->head_dim, Wm = cfg->window - 1;
+  for (int32_t r = 0; r < b->batch; ++r)
+    for (int j = 0; j < Wm; ++j) {
+      const int64_t p = (int64_t)b->ctx_len[r] - Wm + j;
+      for (int kv = 0; kv < 2; ++kv)
+        for (int h = 0; h < Hkv; ++h) {
+          uint16_t* dst = buf + ((((int64_t)r * Wm + j) * 2 + kv) * Hkv + h) * D;
+          if (p < 0) {
+            for (int d = 0; d < D; ++d) dst[d] = 0;
+            continue;
+          }
+          int64_t page;
+          int32_t slot;
+          int rc = orc_locate(cfg, 1, b, r, p, &page, &slot);
+          if (rc != ORC_OK) return rc;
+          if (page < 0 || page >= L->num_pages) return ORC_ERR_RANGE;
+          const int64_t off = elem_offset(L, page, kv, h, slot);
+          for (int d = 0; d < D; ++d) dst[d] = L->pool[off + d * L->stride_d];
+        }
+    }
+  return ORC_OK;
+}
+
+int orc_window_scatter(const orc_config* cfg, const orc_layer* L, const orc_batch* b, const uint16_t* buf) {
+  const int Hkv = cfg->num_kv_heads, D = cfg->head_dim, Wm = cfg->window - 1;
+  for (int32_t r = 0; r < b->batch; ++r)
+    for (int j = 0; j < Wm; ++j) {
+      const int64_t p = (int64_t)b->ctx_len[r] - Wm + j;
+      if (p < 0) continue;
+      int64_t page;
+      int32_t slot;
+      int rc = orc_locate(cfg, 1, b, r, p, &page, &slot);
+      if (rc != ORC_OK) return rc;
+      if (page < 0 || page >= L->num_pages) return ORC_ERR_RANGE;
+      for (int kv = 0; kv < 2; ++kv)
+        for (int h = 0; h < Hkv; ++h) {
+          const uint16_t* src = buf + ((((int64_t)r * Wm + j) * 2 + kv) * Hkv + h) * D;
+          const int64_t off = elem_offset(L, page, kv, h, slot);
+          for (int d = 0; d < D; ++d) L->pool[off + d * L->stride_d] = src[d];
+        }
+    }
+  return ORC_OK;
 }

@@ -79,6 +79,10 @@ def _load():
         lib.orc_kv_append.restype = C.c_int
         lib.orc_attention.restype = C.c_int
         lib.orc_step_advance.restype = C.c_int
+        lib.orc_window_safe_len.restype = C.c_int64
+        lib.orc_window_safe_len.argtypes = [C.c_int64, C.c_int32, C.c_void_p]
+        lib.orc_window_gather.restype = C.c_int
+        lib.orc_window_scatter.restype = C.c_int
         lib.orc_attended_keys.restype = C.c_int64
         lib.orc_attended_keys.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
         _lib = lib
@@ -235,6 +239,29 @@ def step_advance(cfg: OracleConfig, ctx_len: np.ndarray, ring_head: np.ndarray, 
 def attended_keys(cfg: OracleConfig, is_swa: bool, p: int) -> int:
     cc = cfg.c()
     return int(_load().orc_attended_keys(C.byref(cc), C.c_int32(int(is_swa)), C.c_int64(p)))
+
+
+def window_safe_len(match_len: int, window: int, swa_valid) -> int:
+    """Largest hit length <= match_len whose tail still has valid SWA slots (uint8 mask per donor position)."""
+    v = np.ascontiguousarray(swa_valid, dtype=np.uint8)
+    assert v.shape[0] >= match_len
+    return int(_load().orc_window_safe_len(int(match_len), int(window), C.c_void_p(v.ctypes.data)))
+
+
+def window_gather(cfg: OracleConfig, layer: OracleLayer, batch: OracleBatch) -> np.ndarray:
+    """Compact copy [B][W-1][2][Hkv][D] of the cached positions the next token's window needs."""
+    buf = np.zeros((batch.batch, cfg.window - 1, 2, cfg.num_kv_heads, cfg.head_dim), dtype=np.uint16)
+    cc, cl, cb = cfg.c(), layer.c(), batch.c()
+    _check(_load().orc_window_gather(C.byref(cc), C.byref(cl), C.byref(cb), C.c_void_p(buf.ctypes.data)), "window_gather")
+    return buf
+
+
+def window_scatter(cfg: OracleConfig, layer: OracleLayer, batch: OracleBatch, buf: np.ndarray):
+    """Write a compact window buffer into the ring slots of the batch (in place)."""
+    buf = _u16(buf)
+    assert buf.shape == (batch.batch, cfg.window - 1, 2, cfg.num_kv_heads, cfg.head_dim)
+    cc, cl, cb = cfg.c(), layer.c(), batch.c()
+    _check(_load().orc_window_scatter(C.byref(cc), C.byref(cl), C.byref(cb), C.c_void_p(buf.ctypes.data)), "window_scatter")
 
 
 def num_threads() -> int:
