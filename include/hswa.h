@@ -195,6 +195,29 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
                               const void* k_new, const void* v_new, int32_t fuse_append, void* out, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* SWA-aware prefix reuse helpers (paper Sec. 3.1.3 "SWA-Aware Prefix Cache Tree", Sec. 3.1.1 "Data movement",
+ * Sec. 3.1.2 layerwise prefetch).
+ *
+ * hswa_window_safe_len: pure host arithmetic.  A donor matches a new request on its first match_len tokens; its
+ * SWA KV survives only where swa_valid[i] != 0 (host array of at least match_len bytes).  Returns the largest hit
+ * length L <= match_len such that every position in [max(0, L - (W - 1)), L) is valid, i.e. the cached keys the
+ * next token's window needs are all there (0 is always safe; a NULL mask means nothing is valid).
+ *
+ * hswa_swa_window_gather / _scatter: move ONLY the W - 1 cached positions the next token's window needs between
+ * the rings of an SWA layer and a compact buffer bf16 [B][W-1][2 (K,V)][Hkv][D]; entry j of request r is position
+ * ctx_len[r] - (W - 1) + j.  Gather reads the rings (positions below 0 become zeros); scatter writes the ring
+ * slots those positions map to under batch->ring_head / ring_table (positions below 0 are skipped) and touches
+ * nothing else.  `buf` is device memory or pinned host memory (16-byte aligned): gather + scatter with a host
+ * buffer is the offload / loadback of a request's SWA state, scatter into a fresh ring seeds it after a prefix
+ * hit.  (W - 1) * 4 * Hkv * D bytes per request and layer move instead of the whole context.  Layer must be an
+ * SWA layer (HSWA_ERR_INVALID_ARG otherwise); asynchronous on `stream`, so a copy stream can load layer l + 1
+ * while layer l computes. */
+int64_t hswa_window_safe_len(int64_t match_len, int32_t window, const uint8_t* swa_valid);
+hswa_status hswa_swa_window_gather(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, void* buf,
+                                   void* stream);
+hswa_status hswa_swa_window_scatter(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* buf,
+                                    void* stream);
+
 /* Step advance, once per step after all layers: ctx_len[r] += n[r], ring_head[r] = (ring_head[r] + n[r])
  * mod C.  ctx_len, ring_head: device int32 [B], updated in place.  q_indptr: device or NULL (n = 1). */
 hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,

@@ -25,6 +25,7 @@ HSWA_ERR_TIMEOUT = 6
 EXPORTS = [
     "hswa_create", "hswa_destroy", "hswa_workspace_bytes", "hswa_validate_batch", "hswa_kv_append",
     "hswa_decode_attn", "hswa_decode_attn_mtp", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
+    "hswa_window_safe_len", "hswa_swa_window_gather", "hswa_swa_window_scatter",
 ]
 
 
@@ -93,6 +94,12 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_prefill_attn.restype = C.c_int
     lib.hswa_prefill_attn.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp, vp, i32, vp, vp, vp,
                                       sz, vp]
+    lib.hswa_window_safe_len.restype = C.c_int64
+    lib.hswa_window_safe_len.argtypes = [C.c_int64, i32, vp]
+    lib.hswa_swa_window_gather.restype = C.c_int
+    lib.hswa_swa_window_gather.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp]
+    lib.hswa_swa_window_scatter.restype = C.c_int
+    lib.hswa_swa_window_scatter.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp]
     lib.hswa_step_advance.restype = C.c_int
     lib.hswa_step_advance.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.hswa_get_async_error.restype = C.c_int
@@ -234,6 +241,29 @@ def hswa_prefill_attn(h: Handle, layer: Layer, batch: Batch, q, k_new, v_new, fu
     _check(load().hswa_prefill_attn(h.ptr, C.byref(layer.c), C.byref(batch.c), _ptr(q), _ptr(k_new), _ptr(v_new),
                                     int(bool(fuse_append)), _ptr(out), _ptr(lse), _ptr(workspace), ws_bytes,
                                     _stream()), "hswa_prefill_attn")
+
+
+def hswa_window_safe_len(match_len: int, window: int, swa_valid) -> int:
+    """Largest usable hit length given the donor's per-position SWA validity (any uint8 buffer / numpy array)."""
+    import numpy as np
+    v = np.ascontiguousarray(swa_valid, dtype=np.uint8)
+    assert v.shape[0] >= match_len
+    return int(load().hswa_window_safe_len(int(match_len), int(window), C.c_void_p(v.ctypes.data)))
+
+
+def _any_ptr(t: torch.Tensor):
+    assert t.is_contiguous() and (t.is_cuda or t.is_pinned()), "buffer must be a CUDA tensor or pinned host memory"
+    return C.c_void_p(t.data_ptr())
+
+
+def hswa_swa_window_gather(h: Handle, layer: Layer, batch: Batch, buf: torch.Tensor):
+    _check(load().hswa_swa_window_gather(h.ptr, C.byref(layer.c), C.byref(batch.c), _any_ptr(buf), _stream()),
+           "hswa_swa_window_gather")
+
+
+def hswa_swa_window_scatter(h: Handle, layer: Layer, batch: Batch, buf: torch.Tensor):
+    _check(load().hswa_swa_window_scatter(h.ptr, C.byref(layer.c), C.byref(batch.c), _any_ptr(buf), _stream()),
+           "hswa_swa_window_scatter")
 
 
 def hswa_step_advance(h: Handle, batch: int, ctx_len: torch.Tensor, ring_head: torch.Tensor, q_indptr=None):

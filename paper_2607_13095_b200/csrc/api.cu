@@ -489,6 +489,41 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
   return HSWA_OK;
 }
 
+static hswa_status window_move(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, void* buf, int gather,
+                               void* stream) {
+  hswa_status st = check_common(h, layer, b);
+  if (st != HSWA_OK) return st;
+  h->chain_ok = 0;
+  if (!layer->is_swa) return HSWA_ERR_INVALID_ARG;
+  if (b->batch == 0 || h->cfg.window <= 1) return HSWA_OK;
+  if (!buf || !aligned16(buf)) return HSWA_ERR_INVALID_ARG;
+  return hswa_launch_window_move(model_params(h), batch_params(b), static_cast<__nv_bfloat16*>(layer->pool), layer->num_pages,
+                                 static_cast<__nv_bfloat16*>(buf), gather, h->err, (cudaStream_t)stream) == cudaSuccess
+             ? HSWA_OK
+             : HSWA_ERR_CUDA;
+}
+
+hswa_status hswa_swa_window_gather(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, void* buf, void* stream) {
+  return window_move(h, layer, b, buf, 1, stream);
+}
+
+hswa_status hswa_swa_window_scatter(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, const void* buf,
+                                    void* stream) {
+  return window_move(h, layer, b, const_cast<void*>(buf), 0, stream);
+}
+
+int64_t hswa_window_safe_len(int64_t match_len, int32_t window, const uint8_t* swa_valid) {
+  if (match_len <= 0 || window <= 1 || !swa_valid) return match_len > 0 && window <= 1 ? match_len : 0;
+  // run[i] = number of consecutive valid positions ending at i; L is safe iff run[L - 1] >= min(L, W - 1)
+  int64_t best = 0, run = 0;
+  for (int64_t i = 0; i < match_len; ++i) {
+    run = swa_valid[i] ? run + 1 : 0;
+    const int64_t L = i + 1, need = L < window - 1 ? L : window - 1;
+    if (run >= need) best = L;
+  }
+  return best;
+}
+
 hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
                               const int32_t* q_indptr, void* stream) {
   if (h) h->chain_ok = 0;

@@ -71,6 +71,45 @@ __global__ void __launch_bounds__(256) append_ring_kernel(const AppendParams p) 
   *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
 }
 
+// Window-only data movement (paper Sec. 3.1.1 "cross-tier transfers move only valid window data", Sec. 3.1.2
+// layerwise loadback, Sec. 3.1.3 ring seeding after a prefix hit): the W - 1 cached positions the next token's
+// window needs, between a request's ring and a compact buffer [B][W-1][2][Hkv][D].  GATHER: ring -> buffer
+// (positions below 0 become zeros); otherwise buffer -> ring (positions below 0 are skipped).  One thread per
+// 16-byte chunk; blockIdx.y = request.  The buffer may be device memory or pinned host memory.
+template <bool GATHER>
+__global__ void __launch_bounds__(256) window_move_kernel(ModelParams M, BatchParams b, __nv_bfloat16* pool, int64_t num_pages,
+                                                          __nv_bfloat16* buf, int32_t* err) {
+  const int chunks_per_row = M.D / 8;
+  const int chunks_per_tok = 2 * M.Hkv * chunks_per_row;
+  const int Wm = M.W - 1;
+  const int r = blockIdx.y;
+  const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid >= Wm * chunks_per_tok) return;
+  const int j = gid / chunks_per_tok;
+  int c = gid % chunks_per_tok;
+  const int kv = c / (M.Hkv * chunks_per_row);
+  c -= kv * M.Hkv * chunks_per_row;
+  const int kh = c / chunks_per_row;
+  const int ch = c % chunks_per_row;
+  const int pos = b.ctx_len[r] - Wm + j;
+  uint4* slot_in_buf = reinterpret_cast<uint4*>(buf + ((((int64_t)r * Wm + j) * 2 + kv) * M.Hkv + kh) * M.D + ch * 8);
+  if (pos < 0) {
+    if (GATHER) *slot_in_buf = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  const int s = math_mod(b.ring_head[r] - Wm + j, M.C);
+  const int page = b.ring_table[(int64_t)r * M.R + s / M.P];
+  if (page < 0 || page >= num_pages) {
+    record_error(err, HSWA_ERR_BOUNDS, r, s / M.P, page);
+    return;
+  }
+  uint4* in_pool = reinterpret_cast<uint4*>(pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + s % M.P) * M.D + ch * 8);
+  if (GATHER)
+    *slot_in_buf = *in_pool;
+  else
+    *in_pool = *slot_in_buf;
+}
+
 __global__ void advance_kernel(ModelParams M, int B, int32_t* ctx_len, int32_t* ring_head, const int32_t* q_indptr) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= B) return;
@@ -140,5 +179,17 @@ cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int
                                  int32_t* err, cudaStream_t s) {
   if (b.B == 0) return cudaSuccess;
   validate_kernel<<<b.B, 128, 0, s>>>(m, b, is_swa, num_pages, err);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_window_move(const ModelParams& m, const BatchParams& b, __nv_bfloat16* pool, int64_t num_pages,
+                                    __nv_bfloat16* buf, int gather, int32_t* err, cudaStream_t s) {
+  const int per_req = (m.W - 1) * 2 * m.Hkv * (m.D / 8);
+  if (b.B == 0 || per_req == 0) return cudaSuccess;
+  dim3 grid((per_req + 255) / 256, b.B);
+  if (gather)
+    window_move_kernel<true><<<grid, 256, 0, s>>>(m, b, pool, num_pages, buf, err);
+  else
+    window_move_kernel<false><<<grid, 256, 0, s>>>(m, b, pool, num_pages, buf, err);
   return cudaGetLastError();
 }

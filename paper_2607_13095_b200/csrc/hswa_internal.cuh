@@ -124,6 +124,8 @@ cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtens
                                            const PrefillParams& p, int first_tok, cudaStream_t s);
 cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,
                                 const int32_t* q_indptr, cudaStream_t s);
+cudaError_t hswa_launch_window_move(const ModelParams& m, const BatchParams& b, __nv_bfloat16* pool, int64_t num_pages,
+                                    __nv_bfloat16* buf, int gather, int32_t* err, cudaStream_t s);
 cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
                                  int32_t* err, cudaStream_t s);
 

@@ -455,3 +455,42 @@ def test_decode_mtp(d, nq, is_swa):
     assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
     orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
     assert np.array_equal(to_host_bits(pool), ol.pool)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# window-only data movement for SWA prefix reuse
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(4, 64, 16, 1), dims(2, 128, 32, 3, W=33)], ids=str)
+@pytest.mark.parametrize("host_buf", [False, True])
+def test_window_gather_scatter(d, host_buf):
+    W, C = d.window, d.ring_slots
+    ctx = [0, 1, W - 2, W - 1, W, C - 1, C + 1, 3 * C + 5]
+    B = len(ctx)
+    donor = build_scenario(d, ctx, [1] * B, seed=70)
+    h = make_handle(d)
+    layer = hb.Layer(to_dev_bf16(donor.swa_pool), True)
+    shape = (B, W - 1, 2, d.num_kv_heads, d.head_dim)
+    buf = torch.full(shape, 7.0, dtype=torch.bfloat16)
+    buf = buf.pin_memory() if host_buf else buf.cuda()
+    hb.hswa_swa_window_gather(h, layer, dev_batch(donor.tables, True), buf)
+    check_no_async_error(h)
+    ref = orc.window_gather(donor.cfg, donor.layer(True), donor.batch())
+    assert np.array_equal(to_host_bits(buf.cuda()), ref)
+    # seed fresh rings (other pages, other heads) from the buffer: pool bytes must equal the oracle's scatter
+    fresh = wl.make_tables(d, ctx, [1] * B, seed=71)
+    from helpers import poison_pool
+    dst_pool = to_dev_bf16(poison_pool(fresh.num_ring_pages, d))
+    dst = hb.Layer(dst_pool, True)
+    hb.hswa_swa_window_scatter(h, dst, dev_batch(fresh, True), buf)
+    check_no_async_error(h)
+    odst = orc.OracleLayer(poison_pool(fresh.num_ring_pages, d), True)
+    ob = orc.OracleBatch(fresh.ctx_len, fresh.block_table, fresh.ring_table, fresh.ring_head)
+    orc.window_scatter(donor.cfg, odst, ob, ref)
+    assert np.array_equal(to_host_bits(dst_pool), odst.pool)
+    # a decode step on the seeded rings reproduces the donor's output
+    out = torch.zeros((B, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    hb.hswa_decode_attn(h, dst, dev_batch(fresh, True), to_dev_bf16(donor.q), to_dev_bf16(donor.k_new), to_dev_bf16(donor.v_new),
+                        out, None, None)
+    want, _ = orc.attention(donor.cfg, donor.layer(True), donor.batch(), donor.q, donor.k_new, donor.v_new)
+    assert np.abs(out.cpu().numpy() - want).max() <= TOL
+    with pytest.raises(hb.HswaError):
+        hb.hswa_swa_window_gather(h, hb.Layer(to_dev_bf16(donor.full_pool), False), dev_batch(donor.tables, True), buf)

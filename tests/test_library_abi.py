@@ -59,3 +59,16 @@ def test_null_handle_paths():
     assert lib.hswa_workspace_bytes(None, 4, 4, 100) == 0
     assert lib.hswa_step_advance(None, 1, None, None, None, None) == hb.HSWA_ERR_INVALID_ARG
     lib.hswa_destroy(None)
+
+
+def test_window_safe_len_host():
+    import numpy as np
+    from oracle import hswa_oracle as orc
+    rng = np.random.default_rng(1)
+    for W in (1, 2, 4, 128):
+        for _ in range(200):
+            n = int(rng.integers(1, 400))
+            valid = (rng.random(n) < 0.9).astype(np.uint8)
+            valid[: int(rng.integers(0, n))] = rng.integers(0, 2)
+            m = int(rng.integers(0, n + 1))
+            assert hb.hswa_window_safe_len(m, W, valid) == orc.window_safe_len(m, W, valid)
