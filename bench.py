@@ -34,7 +34,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep", "prefetch"])
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
@@ -385,6 +385,72 @@ def run_prefix_sweep(args, torch, device, peaks):
                               "about 0.12x at a 1M prefix (unnamed GPU), attention alone falls further"}))
 
 
+def run_layerwise_prefetch(args, torch, device):
+    """Paper Sec. 3.1.2 (layerwise KVCache prefetch): the SWA state of every request lives in pinned host memory
+    (W - 1 tokens per request and SWA layer: the only part a resumed request needs) and is loaded back layer by
+    layer.  Times one config-5-shaped decode step (70 layers, batch 16) three ways: state already on the device;
+    loadback of layer l right before layer l on the compute stream; loadback on a copy stream running ahead of
+    the compute stream, gated per layer by events."""
+    from paper_2607_13095_b200 import binding as hb
+    w = make_workload("cfg5", layers=args.layers or 70, batch=args.batch)
+    bench = DecodeBench(w, 8, device)
+    d, t = w.dims, bench.t
+    swa = [i for i, s_ in enumerate(w.layer_is_swa) if s_]
+    shape = (t.batch, d.window - 1, 2, d.num_kv_heads, d.head_dim)
+    host = {}
+    for i in swa:  # offload: gather each SWA layer's windows into pinned host memory
+        host[i] = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
+        hb.hswa_swa_window_gather(bench.h, bench.layers[i], bench.batch, host[i])
+    torch.cuda.synchronize()
+    copy_stream = torch.cuda.Stream(device=device, priority=-1)
+    main = torch.cuda.current_stream()
+    # device staging tiles: the DMA engine brings a layer's windows over PCIe, a small kernel scatters them
+    staging = {i: torch.empty(shape, dtype=torch.bfloat16, device=device) for i in swa}
+
+    def layer_call(i):
+        hb.hswa_decode_attn(bench.h, bench.layers[i], bench.batch, bench.q[i], bench.k_new[i], bench.v_new[i], bench.out[i],
+                            None, bench.ws)
+
+    def step_resident():
+        for i in range(len(bench.layers)):
+            layer_call(i)
+
+    def step_serial():
+        for i in range(len(bench.layers)):
+            if i in host:
+                hb.hswa_swa_window_scatter(bench.h, bench.layers[i], bench.batch, host[i])
+            layer_call(i)
+
+    def step_overlapped():
+        start = torch.cuda.Event()
+        start.record(main)
+        events = {}
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(start)  # the previous step has stopped reading the rings
+            for i in swa:
+                staging[i].copy_(host[i], non_blocking=True)
+                hb.hswa_swa_window_scatter(bench.h, bench.layers[i], bench.batch, staging[i])
+                events[i] = torch.cuda.Event()
+                events[i].record(copy_stream)
+        for i in range(len(bench.layers)):
+            if i in events:
+                main.wait_event(events[i])
+            layer_call(i)
+
+    res = {}
+    for name, fn in (("resident", step_resident), ("loadback_serial", step_serial), ("loadback_layerwise", step_overlapped)):
+        res[name + "_ms"] = time_events(torch, fn, 3, args.steps if args.steps < 50 else 10)
+    st = hb.hswa_get_async_error(bench.h)
+    if st[0] != hb.HSWA_OK:
+        raise SystemExit(f"device error word set: {st}")
+    bytes_per_step = len(swa) * int(np.prod(shape)) * 2
+    print(json.dumps({"metric": "decode_step_ms_with_swa_loadback", "unit": "ms", "value": res["loadback_layerwise_ms"], **res,
+                      "n_gpus": 1, "higher_is_better": False, "data": "synthetic", "dtype": "bf16",
+                      "config": {"workload": w.name, "layers": len(w.layer_is_swa), "batch": t.batch},
+                      "h2d_bytes_per_step": bytes_per_step,
+                      "full_kv_bytes_if_not_windowed": int(t.ctx_len.astype(np.int64).sum()) * d.kv_bytes_per_token * len(swa)}))
+
+
 def run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks):
     """--workload cfg3: the chunked-prefill block as the measured workload (value = attention TFLOP/s of the
     whole 1 Full + 6 SWA block, fused append included)."""
@@ -479,6 +545,9 @@ def main():
     hb.load()
     peaks = measured_peaks()
 
+    if args.workload == "prefetch":
+        run_layerwise_prefetch(args, torch, device)
+        return
     if args.workload == "prefix_sweep":
         run_prefix_sweep(args, torch, device, peaks)
         return
