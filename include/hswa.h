@@ -18,7 +18,13 @@
  *   - Host-detectable misuse returns a status at once and launches nothing.  Device-detectable misuse
  *     (hswa_validate_batch; bounded waits inside kernels) is recorded in the error word, the offending
  *     access is skipped, and the kernel returns normally: nothing traps, asserts or spins without bound.
- *   - No global mutable state; a handle may be used from one thread at a time.
+ *   - Within a step the library may overlap consecutive fused decode calls issued through one handle on one
+ *     stream (programmatic dependent launch): a later kernel reads the batch arrays and its layer's pool while
+ *     the earlier one drains, and waits before touching q, k_new, v_new or its outputs.  This relies on the
+ *     contract below that the batch arrays are constant during a step and that only this library writes the
+ *     pools; any other call on the handle (append, prefill, advance, error read) ends the overlap.
+ *   - No global mutable state except the static scratch of hswa_decode_attn_static_ws; a handle may be used
+ *     from one thread at a time.
  *
  * Symbols (bf16 everywhere KV or Q are stored):
  *   Hq, Hkv query / KV heads, G = Hq / Hkv (query head h uses KV head h / G), D head_dim, P page_size,

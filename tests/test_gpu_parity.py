@@ -494,3 +494,66 @@ def test_window_gather_scatter(d, host_buf):
     assert np.abs(out.cpu().numpy() - want).max() <= TOL
     with pytest.raises(hb.HswaError):
         hb.hswa_swa_window_gather(h, hb.Layer(to_dev_bf16(donor.full_pool), False), dev_batch(donor.tables, True), buf)
+
+
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(12))
+def test_random_shapes_stress(seed):
+    """Seeded random shapes, lengths and layer kinds through prefill, decode, multi-token decode and cascade."""
+    rng = np.random.default_rng(1000 + seed)
+    D = int(rng.choice([64, 128]))
+    P = int(rng.choice([16, 32, 64]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.choice([1, 2, 3]))
+    W = int(rng.choice([128, 128, 128, 64, 17]))
+    d = dims(G, D, P, Hkv, W=W)
+    B = int(rng.integers(1, 9))
+    big = rng.random() < 0.3
+    ctx = [int(x) for x in rng.integers(0, 6000 if big else 700, B)]
+    is_swa = bool(rng.integers(0, 2))
+    kind = rng.choice(["prefill", "decode", "mtp", "cascade"])
+    if kind == "prefill":
+        q_len = [int(x) for x in rng.integers(0, 500, B)]
+        if sum(q_len) == 0:
+            q_len[0] = 1
+        sc = build_scenario(d, ctx, q_len, seed=seed)
+        err, lerr = run_prefill(sc, is_swa)
+    elif kind == "decode":
+        sc = build_scenario(d, ctx, [1] * B, seed=seed)
+        err, lerr = run_decode(sc, is_swa, bool(rng.integers(0, 2)))
+    elif kind == "mtp":
+        nq = int(rng.integers(2, 5))
+        if is_swa and nq > d.ring_slots - W + 1:
+            nq = 2
+        sc = build_scenario(d, ctx, [nq] * B, seed=seed, ring_keep=d.ring_slots)
+        t = sc.tables
+        h = make_handle(d)
+        pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+        b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None,
+                     max_q_len=1, total_q=B, max_ctx_len=t.max_ctx_len)
+        out = torch.zeros((B * nq, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+        lse = torch.zeros((B * nq, d.num_q_heads), dtype=torch.float32, device="cuda")
+        ws = torch.empty(hb.hswa_workspace_bytes(h, B, B * nq, t.max_ctx_len + nq) + 256, dtype=torch.uint8, device="cuda")
+        hb.hswa_decode_attn_mtp(h, hb.Layer(pool, is_swa), b, nq, to_dev_bf16(sc.q), to_dev_bf16(sc.k_new),
+                                to_dev_bf16(sc.v_new), out, lse, ws)
+        check_no_async_error(h)
+        ol = sc.layer(is_swa)
+        ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+        orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+        assert np.array_equal(to_host_bits(pool), ol.pool)
+        err, lerr = np.abs(out.cpu().numpy() - ref).max(), np.abs(lse.cpu().numpy() - ref_lse).max()
+    else:
+        prefix = P * int(rng.integers(1, 12))
+        ctx = [prefix + c for c in ctx]
+        sc = build_scenario(d, ctx, [1] * B, seed=seed, shared_prefix_tokens=prefix)
+        t = sc.tables
+        h = make_handle(d)
+        pool = to_dev_bf16(sc.swa_pool if is_swa else sc.full_pool)
+        out = torch.zeros((B, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+        lse = torch.zeros((B, d.num_q_heads), dtype=torch.float32, device="cuda")
+        hb.hswa_decode_attn_shared_prefix(h, hb.Layer(pool, is_swa), dev_batch(t, True), prefix, to_dev_bf16(sc.q),
+                                          to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new), out, lse, workspace_for(h, t))
+        check_no_async_error(h)
+        ref, ref_lse = orc.attention(sc.cfg, sc.layer(is_swa), sc.batch(), sc.q, sc.k_new, sc.v_new)
+        err, lerr = np.abs(out.cpu().numpy() - ref).max(), np.abs(lse.cpu().numpy() - ref_lse).max()
+    assert err <= TOL and lerr <= TOL, (kind, d, is_swa, err, lerr)
