@@ -16,21 +16,16 @@ __device__ __forceinline__ int find_request(const BatchParams& b, int t) {
   return lo;
 }
 
-// One thread moves one 16-byte chunk of one (token, K|V, head) row of a Full layer.
+// Full layer: one warp moves the K (or V) rows of one token, all KV heads: Hkv * D * 2 bytes, up to four
+// 16-byte chunks per lane in flight at once.
 __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
   const ModelParams& M = p.m;
   const int chunks_per_row = M.D / 8;
-  const int chunks_per_tok = 2 * M.Hkv * chunks_per_row;
-  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t total = (int64_t)p.total_q * chunks_per_tok;
-  if (gid >= total) return;
-  const int t = (int)(gid / chunks_per_tok);
-  int c = (int)(gid % chunks_per_tok);
-  const int kv = c / (M.Hkv * chunks_per_row);
-  c -= kv * M.Hkv * chunks_per_row;
-  const int kh = c / chunks_per_row;
-  const int ch = c % chunks_per_row;
-
+  const int chunks = M.Hkv * chunks_per_row;  // 16-byte chunks of one token's K (or V)
+  const int64_t wid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (wid >= (int64_t)p.total_q * 2) return;
+  const int t = (int)(wid >> 1), kv = (int)(wid & 1);
   const int r = p.uniform_n > 0 ? t / p.uniform_n : find_request(p.b, t);
   const int t0 = p.uniform_n > 0 ? r * p.uniform_n : (p.b.q_indptr ? p.b.q_indptr[r] : r);
   const int pos = p.b.ctx_len[r] + (t - t0);
@@ -39,9 +34,24 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
   const int page = p.b.block_table[(int64_t)r * p.b.max_blocks + blk];
   const int slot = pos % M.P;
   if (page < 0 || page >= p.num_pages) return;
-  const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)t * M.Hkv + kh) * M.D + ch * 8;
-  __nv_bfloat16* dst = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + slot) * M.D + ch * 8;
-  *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + (int64_t)t * M.Hkv * M.D;
+  __nv_bfloat16* dst = p.pool + (((int64_t)page * 2 + kv) * M.Hkv * M.P + slot) * M.D;  // head 0 of this (page, K|V)
+  for (int c0 = lane; c0 < chunks; c0 += 128) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + 32 * u;
+      if (c < chunks) v[u] = *reinterpret_cast<const uint4*>(src + c * 8);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + 32 * u;
+      if (c < chunks) {
+        const int kh = c / chunks_per_row, ch = c % chunks_per_row;
+        *reinterpret_cast<uint4*>(dst + (int64_t)kh * M.P * M.D + ch * 8) = v[u];
+      }
+    }
+  }
 }
 
 // SWA layer: only the last min(n, C) tokens of a request survive on its ring (later writes win), so the grid
@@ -162,8 +172,8 @@ cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s) {
     dim3 grid((per_req + 255) / 256, p.b.B);
     append_ring_kernel<<<grid, 256, 0, s>>>(p);
   } else {
-    const int64_t total = (int64_t)p.total_q * chunks_per_tok;
-    append_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(p);
+    const int64_t warps = (int64_t)p.total_q * 2;
+    append_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, s>>>(p);
   }
   return cudaGetLastError();
 }
