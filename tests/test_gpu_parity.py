@@ -557,3 +557,31 @@ def test_random_shapes_stress(seed):
         ref, ref_lse = orc.attention(sc.cfg, sc.layer(is_swa), sc.batch(), sc.q, sc.k_new, sc.v_new)
         err, lerr = np.abs(out.cpu().numpy() - ref).max(), np.abs(lse.cpu().numpy() - ref_lse).max()
     assert err <= TOL and lerr <= TOL, (kind, d, is_swa, err, lerr)
+
+
+@pytest.mark.parametrize("sm_scale", [1.0, 3.0])
+def test_peaked_softmax_exercises_lazy_rescale(sm_scale):
+    """Large score scale: row maxima keep growing from tile to tile by more than the 2^8 slack of the lazy
+    rescale, so the O-rescale path of the tcgen05 kernels (and the split combine with far-apart maxima) runs."""
+    d = dims(8, 128, 64, 1)
+    sc = build_scenario(d, [3000, 0, 777], [300, 520, 129], seed=81, sm_scale=sm_scale)
+    # Nearly one-hot rows: the weight of the dominant key is rounded to bf16 before the PV product (2^-9 relative)
+    # while the row sum keeps fp32, and the output is rounded to bf16 once more; neither averages out over keys
+    # here, so the bound is 2^-8 max|v| instead of the 1e-2 that holds at the model's 1/sqrt(D) scale.
+    vmax = float(np.abs(wl.bits_to_f64(sc.full_pool[:, 1])).max())
+    tol = max(TOL, 2.0 ** -8 * max(vmax, float(np.abs(wl.bits_to_f64(sc.v_new)).max())))
+    for is_swa in (False, True):
+        err, lerr = run_prefill(sc, is_swa)
+        assert err <= tol and lerr <= 2 * TOL * max(1.0, sm_scale), (is_swa, err, lerr, tol)
+    prefix = 64 * 40
+    sc = build_scenario(d, [prefix + 5, prefix + 2100, prefix], [1, 1, 1], seed=82, sm_scale=sm_scale, shared_prefix_tokens=prefix)
+    t = sc.tables
+    h = make_handle(d, sm_scale=sm_scale)
+    out = torch.zeros((3, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    hb.hswa_decode_attn_shared_prefix(h, hb.Layer(to_dev_bf16(sc.full_pool), False), dev_batch(t, True), prefix, to_dev_bf16(sc.q),
+                                      to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new), out, None, workspace_for(h, t))
+    check_no_async_error(h)
+    ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
+    assert np.abs(out.cpu().numpy() - ref).max() <= TOL
+    err, lerr = run_decode(build_scenario(d, [9000, 130], [1, 1], seed=83, sm_scale=sm_scale), False, True)
+    assert err <= TOL, err
