@@ -5,13 +5,16 @@
 //
 // One thread block = 128 query tokens x 2 query heads of one GQA group (two 128-row Q tiles that share every
 // K/V tile and every mask).  Warp roles:
-//   warps 0-7   softmax for Q tile 0: TMEM lane = row; two warps share each 32-row lane quadrant and take 64 key
-//               columns each, exchanging partial row maxima / sums through shared memory
-//   warps 8-15  softmax for Q tile 1
-//   warp  16    TMA producer: Q once, then 128-key K and V tiles through two 2-stage rings
-//   warp  17    MMA issuer: S_i = Q_i K^T (SS form), O_i += P_i V (TS form, P read from TMEM where it
-//               overwrites S_i), in the order PV0(j), S0(j+1), PV1(j), S1(j+1) so that one tile's softmax
-//               overlaps the other tile's MMAs
+//   warps 0-3   softmax for Q tile 0: TMEM lane = row = thread; a thread holds the 128 scores of its row in
+//               registers, so row maxima and sums need no exchange
+//   warps 4-7   softmax for Q tile 1
+//   warp  8     TMA producer: Q once, then 128-key K and V tiles through two 2-stage rings whose slots are
+//               released separately (K right after the S MMAs, V after both tiles' PV MMAs)
+//   warps 9,10  MMA issuers, one per Q tile: S_i = Q_i K^T (SS form), O_i += P_i V (TS form, P read from TMEM
+//               where it overwrites S_i).  They take turns, [PV0(j), S0(j+1)] [PV1(j), S1(j+1)] ..., so that one
+//               tile's softmax overlaps the other tile's MMAs; while one holds the turn, the other polls the
+//               mbarriers of its next group (an mbarrier poll costs 100-200 cycles while the tensor cores
+//               saturate shared memory, and a single issuer spent a third of its time in them)
 // TMEM columns: S0 0-127, S1 128-255, O0 256-383, O1 384-511 (all fp32; P_i = bf16 pairs in the first 64
 // columns of S_i).  O is rescaled lazily: only when a row maximum grows by more than 2^8.
 //
@@ -31,7 +34,7 @@ constexpr int PG = 64;                // page size
 constexpr int HALF_BYTES = 128 * 128; // [128 rows][128 B]: one 64-element half of a 128-row tile
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int KV_STAGES = 2;
-constexpr int NUM_THREADS = 576;  // 16 softmax warps + producer + MMA issuer
+constexpr int NUM_THREADS = 352;  // 8 softmax warps + producer + one MMA issuer per Q tile
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                  // 2 Q tiles
@@ -45,7 +48,7 @@ constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [ke
 
 // barrier indices
 enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9,
-       BAR_PFULL = 11 /* [Q tile][first / second half of each warp's columns] */, BAR_OFINAL = 15, NUM_BARS = 16 };
+       BAR_PFULL = 11 /* [Q tile][half of the key columns] */, BAR_OFINAL = 15 /* [Q tile] */, NUM_BARS = 17 };
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -87,6 +90,17 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
   return d;
 }
 
+constexpr int P_PARTS = 2;  // P is posted to the MMA issuer in two halves of 64 keys
+
+// One lane of a converged warp; the rest of the warp skips the guarded statement.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+// Descriptor of the same matrix layout starting `bytes` further on (the start address field holds address / 16).
+__device__ __forceinline__ uint64_t desc_advance(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -116,15 +130,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t* r) {
       "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(addr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};" ::"r"(r[0]),
-      "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
-      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(addr)
-      : "memory");
-}
-
 __device__ __forceinline__ void tmem_st16p(uint32_t addr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
@@ -138,11 +143,15 @@ __device__ __forceinline__ void tmem_st8(uint32_t addr, const uint32_t* r) {
                "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(addr)
                : "memory");
 }
-__device__ __forceinline__ void tmem_ld8(uint32_t addr, uint32_t* r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(addr)
-               : "memory");
+
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(addr)
+      : "memory");
 }
 
 // The sequence of key tiles one block walks: nA cached tiles, then chunk tiles c_lo .. c_lo + nB - 1.
@@ -177,7 +186,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[NUM_BARS];
   __shared__ uint32_t tmem_base_slot;
-  __shared__ float xch[2][2][2][128];  // [parity][Q tile][column half][row]: partial row maxima / sums
+  __shared__ int mma_abort;  // set by an MMA issuer that gave up, read by the other one
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
@@ -214,7 +223,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     h0 = kh * M.G + pair * 2;
     seq = tile_seq(p.is_swa, ctx, b, M.W, M.R);
   }
-  if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;  // an earlier block gave up: do not queue behind it
+  // An earlier block gave up: do not queue behind it.  One thread reads the error word so that the whole block
+  // takes the same decision (the MMA issuers below wait for each other on counted barriers).
+  if (threadIdx.x == 0) mma_abort = *reinterpret_cast<volatile int32_t*>(p.err) != 0;
+  __syncthreads();
+  if (mma_abort) return;
   const int n_tiles = seq.total();
 
   auto bar = [&](int i) { return smem_u32(&bars[i]); };
@@ -223,19 +236,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     mbar_init(bar(BAR_Q), 1);
     for (int s = 0; s < KV_STAGES; ++s) {
       mbar_init(bar(BAR_KFULL + s), 1);
-      mbar_init(bar(BAR_KEMPTY + s), 1);
+      mbar_init(bar(BAR_KEMPTY + s), 2);  // one commit per MMA issuer
       mbar_init(bar(BAR_VFULL + s), 1);
-      mbar_init(bar(BAR_VEMPTY + s), 1);
+      mbar_init(bar(BAR_VEMPTY + s), 2);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_PFULL + 2 * i), 8);  // one arrival per softmax warp
-      mbar_init(bar(BAR_PFULL + 2 * i + 1), 8);
+      for (int q = 0; q < P_PARTS; ++q) mbar_init(bar(BAR_PFULL + P_PARTS * i + q), 4);  // one arrival per softmax warp
     }
     mbar_init(bar(BAR_OFINAL), 1);
+    mbar_init(bar(BAR_OFINAL + 1), 1);
     mbar_fence_init();
   }
-  if (warp == 16) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -245,7 +258,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
-  if (warp == 16) {
+  if (warp == 8) {
     // ======================= TMA producer =======================
     if (lane == 0) {
       tma_prefetch_desc(&tm_pool);
@@ -281,17 +294,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         pg[1] = __shfl_sync(0xffffffffu, pid_cur, i1 & 31);
       }
       if (lane == 0) {
-        if (j >= KV_STAGES) {
-          const uint32_t par = ((j / KV_STAGES) - 1) & 1;
-          if (!mbar_wait(bar(BAR_KEMPTY + stage), par) || !mbar_wait(bar(BAR_VEMPTY + stage), par)) {
-            record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 10);
+        // K and V slots are released separately (K right after the S MMAs that read it, V only after both tiles'
+        // PV MMAs), so each load waits for its own slot: the K tile is on its way a whole step earlier.
+        const uint32_t par = ((j / KV_STAGES) - 1) & 1;
+        const uint32_t dK = sbase + OFF_K + stage * TILE_BYTES, dV = sbase + OFF_V + stage * TILE_BYTES;
+        for (int kv = 0; kv < 2 && ok; ++kv) {
+          const uint32_t full = bar((kv ? BAR_VFULL : BAR_KFULL) + stage);
+          if (j >= KV_STAGES && !mbar_wait(bar((kv ? BAR_VEMPTY : BAR_KEMPTY) + stage), par)) {
+            record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 10 + kv);
             ok = false;
+            break;
           }
-        }
-        if (ok) {
-          const uint32_t dK = sbase + OFF_K + stage * TILE_BYTES, dV = sbase + OFF_V + stage * TILE_BYTES;
-          mbar_arrive_expect_tx(bar(BAR_KFULL + stage), TILE_BYTES);
-          mbar_arrive_expect_tx(bar(BAR_VFULL + stage), TILE_BYTES);
+          mbar_arrive_expect_tx(full, TILE_BYTES);
+          const uint32_t dst = kv ? dV : dK;
           if (j < seq.nA) {
             for (int q = 0; q < 2; ++q) {
               int page = pg[q];
@@ -299,102 +314,130 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
                 record_error(p.err, HSWA_ERR_BOUNDS, r, 2 * j + q, page);
                 page = 0;
               }
-              for (int hf = 0; hf < 2; ++hf) {
-                tma_load_4d(dK + hf * HALF_BYTES + q * PG * 128, &tm_pool, bar(BAR_KFULL + stage), hf * 64, 0, kh, page);
-                tma_load_4d(dV + hf * HALF_BYTES + q * PG * 128, &tm_pool, bar(BAR_VFULL + stage), hf * 64, 0,
-                            M.Hkv + kh, page);
-              }
+              for (int hf = 0; hf < 2; ++hf)
+                tma_load_4d(dst + hf * HALF_BYTES + q * PG * 128, &tm_pool, full, hf * 64, 0, kv * M.Hkv + kh, page);
             }
           } else {
             const int tok = t0 + (seq.c_lo + (j - seq.nA)) * BN;
-            for (int hf = 0; hf < 2; ++hf) {
-              tma_load_3d(dK + hf * HALF_BYTES, &tm_k, bar(BAR_KFULL + stage), hf * 64, kh, tok);
-              tma_load_3d(dV + hf * HALF_BYTES, &tm_v, bar(BAR_VFULL + stage), hf * 64, kh, tok);
-            }
+            for (int hf = 0; hf < 2; ++hf) tma_load_3d(dst + hf * HALF_BYTES, kv ? &tm_v : &tm_k, full, hf * 64, kh, tok);
           }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
     }
-  } else if (warp == 17) {
+  } else if (warp == 9 || warp == 10) {
     // ======================= MMA issuer =======================
-    if (lane == 0) {
+    // The whole warp walks the loop converged (waits, descriptor arithmetic); one elected lane issues.
+    {
       bool ok = mbar_wait(bar(BAR_Q), 0);
+      const uint64_t dQ0 = smem_desc(sbase + OFF_Q, 16), dQ1 = smem_desc(sbase + OFF_Q + TILE_BYTES, 16);
+      const uint64_t dK0 = smem_desc(sbase + OFF_K, 16), dV0 = smem_desc(sbase + OFF_V, HALF_BYTES);
       auto issue_S = [&](int i, int stage) {
         tc_fence_after();
-        const uint32_t aQ = sbase + OFF_Q + i * TILE_BYTES, aK = sbase + OFF_K + stage * TILE_BYTES;
+        const uint64_t dq = i ? dQ1 : dQ0, dk = desc_advance(dK0, stage * TILE_BYTES);
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-          tc_mma_ss(tmem + i * 128, smem_desc(aQ + off, 16), smem_desc(aK + off, 16), IDESC_S, ks > 0);
+          for (int ks = 0; ks < HD / 16; ++ks) {
+            const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+            tc_mma_ss(tmem + i * 128, desc_advance(dq, off), desc_advance(dk, off), IDESC_S, ks > 0);
+          }
+          tc_commit(bar(BAR_SFULL + i));
         }
-        tc_commit(bar(BAR_SFULL + i));
+        __syncwarp();
       };
-      // PV k-steps of one part: warps of column half h post keys 64 h + 32 part + [0, 32) = k-steps 4 h + 2 part + {0, 1}
+      // PV k-steps of one part of the keys, issued as soon as its P columns are posted
+      constexpr int KSTEPS = 8 / P_PARTS;
       auto issue_PV = [&](int i, int stage, int part, bool first) {
         tc_fence_after();
-        const uint32_t aV = sbase + OFF_V + stage * TILE_BYTES;
+        const uint64_t dv = desc_advance(dV0, stage * TILE_BYTES + part * KSTEPS * 2048);
+        const uint32_t tp = tmem + i * 128 + part * KSTEPS * 8;
+        if (elect_one()) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int kk = (q >> 1) * 4 + part * 2 + (q & 1);
-          tc_mma_ts(tmem + 256 + i * 128, tmem + i * 128 + kk * 8, smem_desc(aV + kk * 2048, HALF_BYTES), IDESC_PV,
-                    !(first && part == 0 && q == 0));
+          for (int q = 0; q < KSTEPS; ++q)
+            tc_mma_ts(tmem + 256 + i * 128, tp + q * 8, desc_advance(dv, q * 2048), IDESC_PV, !(first && part == 0 && q == 0));
         }
+        __syncwarp();
       };
+      // One issuer per Q tile, taking turns: [PV0(j), S0(j+1)] [PV1(j), S1(j+1)] [PV0(j+1), ...].  The turn is a
+      // token passed through two named barriers (hardware barriers: no shared-memory round trip), so the order in
+      // the tensor queue is the one that keeps the tiles half a step apart, while each issuer polls the
+      // mbarriers of its next group during the other issuer's turn.  A warp leaves the loop only right after
+      // passing the token, and passes it whenever it finds the abort flag set, so neither can wait forever.
+      const int i = warp - 9;
+      const int tok_in = i == 0 ? 2 : 1, tok_out = i == 0 ? 1 : 2;
+      auto token_wait = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(tok_in) : "memory"); };
+      auto token_pass = [&]() {
+        __threadfence_block();  // the abort flag, if set, is visible to the warp this releases
+        asm volatile("bar.arrive %0, 64;" ::"r"(tok_out) : "memory");
+      };
+      volatile int* abort_flag = &mma_abort;
       if (ok) ok = mbar_wait(bar(BAR_KFULL + 0), 0);
-      if (ok) {
-        issue_S(0, 0);
-        issue_S(1, 0);
-        tc_commit(bar(BAR_KEMPTY + 0));
+      if (i == 1) token_wait();
+      if (!ok) *abort_flag = 1;
+      if (ok && *abort_flag == 0) {
+        issue_S(i, 0);
+        if (elect_one()) tc_commit(bar(BAR_KEMPTY + 0));
+        __syncwarp();
       }
-      for (int j = 0; j < n_tiles && ok; ++j) {
+      token_pass();
+      bool done = !ok || *abort_flag != 0;
+      for (int j = 0; j < n_tiles && !done; ++j) {
         const int stage = j % KV_STAGES, nstage = (j + 1) % KV_STAGES;
         const bool more = j + 1 < n_tiles;
-        ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + 0), j & 1);
-        if (!ok) break;
-        issue_PV(0, stage, 0, j == 0);
-        ok = mbar_wait(bar(BAR_PFULL + 1), j & 1);
-        if (!ok) break;
-        issue_PV(0, stage, 1, false);
-        if (more) {
-          ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
-          if (!ok) break;
-          issue_S(0, nstage);
+        // polled during the other issuer's turn
+        ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + P_PARTS * i), j & 1);
+        if (ok && more) ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
+        token_wait();
+        if (!ok) *abort_flag = 1;
+        if (*abort_flag != 0) {
+          token_pass();
+          break;
         }
-        ok = mbar_wait(bar(BAR_PFULL + 2), j & 1);
-        if (!ok) break;
-        issue_PV(1, stage, 0, j == 0);
-        ok = mbar_wait(bar(BAR_PFULL + 3), j & 1);
-        if (!ok) break;
-        issue_PV(1, stage, 1, false);
-        tc_commit(bar(BAR_VEMPTY + stage));
-        if (more) {
-          issue_S(1, nstage);
-          tc_commit(bar(BAR_KEMPTY + nstage));
+#pragma unroll
+        for (int q = 0; q < P_PARTS; ++q) {
+          if (q > 0 && ok) ok = mbar_wait(bar(BAR_PFULL + P_PARTS * i + q), j & 1);
+          if (ok) issue_PV(i, stage, q, j == 0);
         }
+        if (ok) {
+          if (elect_one()) tc_commit(bar(BAR_VEMPTY + stage));
+          __syncwarp();
+          if (more) {
+            issue_S(i, nstage);
+            if (elect_one()) tc_commit(bar(BAR_KEMPTY + nstage));
+            __syncwarp();
+          }
+        } else {
+          *abort_flag = 1;
+          done = true;
+        }
+        token_pass();
       }
-      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 20);
-      tc_commit(bar(BAR_OFINAL));
+      if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 20 + i);
+      if (elect_one()) tc_commit(bar(BAR_OFINAL + i));
+      __syncwarp();
     }
   } else {
     // ======================= softmax warps =======================
-    // 8 warps per Q tile: warp pair (quad, half) shares the 32 rows of a TMEM lane quadrant and splits the 128
-    // key columns in two, so four softmax warps are resident per scheduler and hide each other's MUFU and
-    // TMEM latencies.  The halves of a row exchange their partial maxima through shared memory.
-    const int i = warp >> 3;                    // Q tile
-    const int quad = warp & 3, half = (warp >> 2) & 1;
+    // 4 warps per Q tile: TMEM lane = row = thread, which holds all 128 scores of its row in registers, so row
+    // maxima and sums need no exchange.  P is written to TMEM in four quarters of 32 keys and posted to the MMA
+    // issuer in two halves; the first half is posted once the third quarter's exponentials are under way,
+    // which hides the TMEM store latency.
+    const int i = warp >> 2;                    // Q tile
+    const int quad = warp & 3;
     const int rr = quad * 32 + lane;            // row in the tile = TMEM lane
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t tS = tmem + lane_addr + i * 128 + half * 64;
-    const uint32_t tP = tmem + lane_addr + i * 128 + half * 32;
-    const uint32_t tO = tmem + lane_addr + 256 + i * 128 + half * 64;
-    const int pair_bar = 1 + i * 4 + quad;      // named barrier of the two warps that share these rows
+    const uint32_t tS = tmem + lane_addr + i * 128;
+    const uint32_t tO = tmem + lane_addr + 256 + i * 128;
     const int ri = b * BM + rr;                 // chunk-relative row
     const int pos = ctx + ri;                   // absolute position
     float m_st = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_SFULL + i), j & 1));  // warp-uniform: TMEM ops are warp-wide
+      if (!ok) {
+        if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 30 + i);
+        break;
+      }
       // visible column interval [lo, hi) of this row in this tile; ring tiles are decided per column
       int lo = 0, hi = BN;
       bool ring_tile = false, masked = false;
@@ -416,69 +459,60 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         }
         masked = (c == b) || p.is_swa;
       }
-      // bit k of (vm_lo, vm_hi) = this thread's column half * 64 + k is visible to this row
-      uint32_t vm_lo = 0xffffffffu, vm_hi = 0xffffffffu;
+      // bit k of vm[w] = column 32 w + k is visible to this row
+      uint32_t vm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
       if (masked) {
-        if (!ring_tile) {
-          int c0 = lo - half * 64, c1 = hi - half * 64;
-          c0 = c0 < 0 ? 0 : (c0 > 64 ? 64 : c0);
-          c1 = c1 < 0 ? 0 : (c1 > 64 ? 64 : c1);
-          const uint64_t below_c1 = c1 >= 64 ? ~0ull : ((1ull << c1) - 1);
-          const uint64_t below_c0 = c0 >= 64 ? ~0ull : ((1ull << c0) - 1);
-          const uint64_t vm = c1 > c0 ? (below_c1 & ~below_c0) : 0ull;
-          vm_lo = (uint32_t)vm;
-          vm_hi = (uint32_t)(vm >> 32);
-        } else {
-          // ring tile: ring page 2j + half; slot -> position it held before the chunk's append
-          uint64_t vm = 0;
-          const int page_in_ring = 2 * j + half;
-          if (page_in_ring < M.R) {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint64_t m64 = 0;
+          if (!ring_tile) {
+            int c0 = lo - hf * 64, c1 = hi - hf * 64;
+            c0 = c0 < 0 ? 0 : (c0 > 64 ? 64 : c0);
+            c1 = c1 < 0 ? 0 : (c1 > 64 ? 64 : c1);
+            const uint64_t below_c1 = c1 >= 64 ? ~0ull : ((1ull << c1) - 1);
+            const uint64_t below_c0 = c0 >= 64 ? ~0ull : ((1ull << c0) - 1);
+            m64 = c1 > c0 ? (below_c1 & ~below_c0) : 0ull;
+          } else {
+            // ring tile: ring page 2j + hf; slot -> position it held before the chunk's append
+            const int page_in_ring = 2 * j + hf;
+            if (page_in_ring < M.R) {
 #pragma unroll 1
-            for (int k = 0; k < 64; ++k) {
-              int off = page_in_ring * PG + k - head;
-              if (off < 0) off += M.C;
-              const int kpos = ctx - M.C + off;
-              if (kpos >= 0 && kpos > pos - M.W) vm |= 1ull << k;
+              for (int k = 0; k < 64; ++k) {
+                int off = page_in_ring * PG + k - head;
+                if (off < 0) off += M.C;
+                const int kpos = ctx - M.C + off;
+                if (kpos >= 0 && kpos > pos - M.W) m64 |= 1ull << k;
+              }
             }
           }
-          vm_lo = (uint32_t)vm;
-          vm_hi = (uint32_t)(vm >> 32);
+          vm[2 * hf] = (uint32_t)m64;
+          vm[2 * hf + 1] = (uint32_t)(m64 >> 32);
         }
       }
-      // this thread's 64 scores: one round trip to TMEM
-      uint32_t v[64];
-      float mx = INFINITY;  // +inf tells the partner warp that this warp gave up
-      if (ok) {
-        tc_fence_after();
-        tmem_ld32(tS, v);
-        tmem_ld32(tS + 32, v + 32);
-        tc_wait_ld();
-        if (masked) {
+      // this thread's 128 scores: one round trip to TMEM
+      uint32_t v[128];
+      tc_fence_after();
+      tmem_ld32(tS, v);
+      tmem_ld32(tS + 32, v + 32);
+      tmem_ld32(tS + 64, v + 64);
+      tmem_ld32(tS + 96, v + 96);
+      tc_wait_ld();
+      if (masked) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            if (!((vm_lo >> k) & 1u)) v[k] = 0xff800000u;  // -inf
-            if (!((vm_hi >> k) & 1u)) v[32 + k] = 0xff800000u;
-          }
-        }
-        float mx4[4];
+        for (int w4 = 0; w4 < 4; ++w4)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) mx4[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
-#pragma unroll
-        for (int k = 8; k < 64; k += 8) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) mx4[c] = max3(mx4[c], __uint_as_float(v[k + 2 * c]), __uint_as_float(v[k + 2 * c + 1]));
-        }
-        mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          for (int k = 0; k < 32; ++k)
+            if (!((vm[w4] >> k) & 1u)) v[32 * w4 + k] = 0xff800000u;  // -inf
       }
-      xch[j & 1][i][half][rr] = mx;
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-      const float other = xch[j & 1][i][half ^ 1][rr];
-      if (!ok || __any_sync(0xffffffffu, other == INFINITY)) {
-        if (lane == 0 && !ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 30 + i);
-        ok = false;
-        break;
+      float mx8[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) mx8[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+#pragma unroll
+      for (int k = 16; k < 128; k += 16) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) mx8[c] = max3(mx8[c], __uint_as_float(v[k + 2 * c]), __uint_as_float(v[k + 2 * c + 1]));
       }
-      mx = fmaxf(mx, other);
+      const float mx = fmaxf(fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5])), fmaxf(mx8[6], mx8[7]));
       const float mx_s = mx * M.scale_log2;
       if (j == 0) {
         m_st = mx_s;
@@ -488,13 +522,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
           const float m_new = grow ? mx_s : m_st;
           const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_st - m_new);
 #pragma unroll 1
-          for (int c8 = 0; c8 < 8; ++c8) {  // small chunks: the 64 scores stay live in registers meanwhile
-            uint32_t w[8];
-            tmem_ld8(tO + c8 * 8, w);
+          for (int c16 = 0; c16 < 8; ++c16) {
+            uint32_t w[16];
+            tmem_ld16(tO + c16 * 16, w);
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 8; ++k) w[k] = __float_as_uint(__uint_as_float(w[k]) * alpha);
-            tmem_st8(tO + c8 * 8, w);
+            for (int k = 0; k < 16; ++k) w[k] = __float_as_uint(__uint_as_float(w[k]) * alpha);
+            tmem_st16p(tO + c16 * 16, w);
           }
           l_run *= alpha;
           m_st = m_new;
@@ -506,10 +540,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       float2 acc[4];
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[c] = make_float2(0.f, 0.f);
-      // Two parts of 32 keys each: the MMA warp starts the PV k-steps of a part as soon as all warps posted it,
-      // so half of the PV MMA overlaps the second part's exponentials.
+      constexpr int QPP = 4 / P_PARTS;  // 32-key quarters per posted part
 #pragma unroll
-      for (int part = 0; part < 2; ++part) {
+      for (int part = 0; part < 4; ++part) {
 #pragma unroll
         for (int k = part * 16; k < part * 16 + 16; ++k) {
           const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
@@ -519,100 +552,94 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
           // costs one more ALU op per key and 6.5 % of the kernel's time; the difference shows only for nearly
           // one-hot rows, where it is bounded by 2^-9 max|v|)
           acc[k & 3] = __fadd2_rn(acc[k & 3], e);
+          if (part > 0 && (part % QPP) == 0 && k == part * 16 + 7) {
+            // post the previous half: its TMEM stores have landed by now, so the wait costs nothing
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_PFULL + P_PARTS * i + part / QPP - 1));  // one arrival per warp
+          }
         }
-        tmem_st16p(tP + part * 16, v + part * 16);
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(BAR_PFULL + 2 * i + part));  // 32 arrivals on one barrier word would serialise
+        tmem_st16p(tS + part * 16, v + part * 16);
+        if (part == 3) {
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(BAR_PFULL + P_PARTS * i + P_PARTS - 1));
+        }
       }
       const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
       l_run += (a01.x + a01.y) + (a23.x + a23.y);
     }
     // ---- epilogue: O / l -> global ----
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFINAL), 0));
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_OFINAL + i), 0));
     if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, b, 40 + i);
     tc_fence_after();
-    // the two halves of a row add up their partial sums (a warp that gave up posts NaN so both halves skip)
-    xch[0][i][half][rr] = ok ? l_run : NAN;
-    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-    const float l_other = xch[0][i][half ^ 1][rr];
-    ok = ok && !__any_sync(0xffffffffu, l_other != l_other);
-    const float l_tot = l_run + l_other;
+    const float l_tot = l_run;
     if constexpr (PREFIX) {
       // partial for the split-K combine: row = (request, head), unnormalised o with its (m, l)
       const int rq = r + 16 * i + (rr >> 3);
       const bool row_ok = ok && rq < p.b.B;
       const int64_t prow = ((int64_t)rq * M.Hq + kh * M.G + (rr & 7)) * p.max_splits + blockIdx.x;
 #pragma unroll 1
-      for (int c2 = 0; c2 < 2; ++c2) {
+      for (int c4 = 0; c4 < 4; ++c4) {
         uint32_t w[32];
-        tmem_ld32(tO + c2 * 32, w);
+        tmem_ld32(tO + c4 * 32, w);
         tc_wait_ld();
         if (row_ok) {
-          float4* dst = reinterpret_cast<float4*>(p.part_o + prow * HD + half * 64 + c2 * 32);
+          float4* dst = reinterpret_cast<float4*>(p.part_o + prow * HD + c4 * 32);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
             dst[k] = make_float4(__uint_as_float(w[4 * k]), __uint_as_float(w[4 * k + 1]), __uint_as_float(w[4 * k + 2]),
                                  __uint_as_float(w[4 * k + 3]));
         }
       }
-      if (row_ok && half == 0) p.part_ml[prow] = make_float2(m_st, l_tot);
+      if (row_ok) p.part_ml[prow] = make_float2(m_st, l_tot);
     } else {
-    const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-    const bool row_ok = ok && ri < n;
-    const int64_t orow = ((int64_t)(t0 + ri) * M.Hq + (h0 + i));
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      const bool row_ok = ok && ri < n;
+      const int64_t orow = ((int64_t)(t0 + ri) * M.Hq + (h0 + i));
 #pragma unroll 1
-    for (int c2 = 0; c2 < 2; ++c2) {
-      uint32_t w[32];
-      tmem_ld32(tO + c2 * 32, w);
-      tc_wait_ld();
-      if (row_ok) {
-        const int col0 = half * 64 + c2 * 32;
-        if (M.out_fp32) {
-          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + col0);
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t w[32];
+        tmem_ld32(tO + c4 * 32, w);
+        tc_wait_ld();
+        if (row_ok) {
+          const int col0 = c4 * 32;
+          if (M.out_fp32) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD + col0);
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
-                                 __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + col0);
+            for (int k = 0; k < 8; ++k)
+              dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
+                                   __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD + col0);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            uint4 u;
-            u.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
-            u.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
-            u.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
-            u.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
-            dst[k] = u;
+            for (int k = 0; k < 4; ++k) {
+              uint4 u;
+              u.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
+              u.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
+              u.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
+              u.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
+              dst[k] = u;
+            }
           }
         }
       }
-    }
-    if (row_ok && half == 0 && p.lse)
-      p.lse[orow] = l_tot > 0.f ? (m_st + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+      if (row_ok && p.lse) p.lse[orow] = l_tot > 0.f ? (m_st + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
   // ---- teardown: everyone is done with TMEM before it is released ----
   tc_fence_before();
   __syncthreads();
-  if (warp == 16) {
+  if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
   }
 }
 
 
-__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(addr)
-      : "memory");
-}
 
 // ---------------------------------------------------------------------------------------------------------
 // SWA layers, tokens whose whole window lies inside the chunk (paper Sec. 2.1: an SWA layer attends to W keys
@@ -1075,7 +1102,6 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       const int tok = i0 + s * SUB + tl;
       const bool row_ok = ok && tok < n;
       const int64_t orow = (int64_t)(t0 + tok) * M.Hq + kh * G + g;
-      const int qb = s % QBUF;
       // Full sub-tiles with bf16 output leave through a shared-memory staging tile and one TMA tensor store; a row-per-thread global store would touch 32 scattered sectors per
       // instruction.  Ragged tails and fp32 output use plain stores.
       const bool staged = tma_out && ok && (i0 + s * SUB + SUB <= n);
