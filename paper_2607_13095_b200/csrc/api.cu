@@ -73,14 +73,15 @@ int plan_max_splits(int split_len, int max_ctx_len) {
   return (int)((kv_len + split_len - 1) / split_len);
 }
 
-// 4-D view of a pool for TMA: {D, P, 2 * Hkv, num_pages}, box {64, P, 1, 1}, 128-byte swizzle.
-hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtensorMap* tm) {
+// 4-D view of a pool for TMA: {D, P, 2 * Hkv, num_pages}, box {64, box_slots, 1, 1} (0: a whole page),
+// 128-byte swizzle.
+hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtensorMap* tm, int box_slots = 0) {
   const hswa_config& c = h->cfg;
   cuuint64_t dims[4] = {(cuuint64_t)c.head_dim, (cuuint64_t)c.page_size, (cuuint64_t)(2 * c.num_kv_heads),
                         (cuuint64_t)layer->num_pages};
   cuuint64_t strides[3] = {(cuuint64_t)c.head_dim * 2, (cuuint64_t)c.head_dim * 2 * c.page_size,
                            (cuuint64_t)c.head_dim * 2 * c.page_size * 2 * c.num_kv_heads};
-  cuuint32_t box[4] = {64, (cuuint32_t)c.page_size, 1, 1};
+  cuuint32_t box[4] = {64, (cuuint32_t)(box_slots > 0 ? box_slots : c.page_size), 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult rc = h->encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, layer->pool, dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -293,7 +294,8 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
     }
   }
   CUtensorMap tm;
-  st = make_pool_map(h, layer, &tm);
+  // SWA layers: the ring kernel loads 16-slot granules, only those that meet the window
+  st = make_pool_map(h, layer, &tm, layer->is_swa ? (h->cfg.page_size < HSWA_RING_GRANULE ? h->cfg.page_size : HSWA_RING_GRANULE) : 0);
   if (st != HSWA_OK) return st;
   // A fused decode that directly follows another fused decode of the same step (same handle, stream and batch
   // arrays) may start early: those kernels never write the batch arrays or another layer's pool.

@@ -42,19 +42,24 @@ struct KeyRange {
   }
 };
 
-// One consumer warp's work on a staged 64-key tile: zero the V rows of invisible keys, S^T = K Q^T, online
-// softmax for the warp's (m, l, O^T) state, O^T += V^T P^T.  (vm0, vm1) is the 64-bit visibility mask of the tile for
-// this warp's query; V rows whose bit in (zm0, zm1) is clear are zeroed (rows no query of the block can see).
-template <int D>
+// One consumer warp's work on a staged 64-key tile: S^T = K Q^T, online softmax for the warp's (m, l, O^T)
+// state, O^T += V^T P^T.  (vm0, vm1) is the 64-bit visibility mask of the tile for this warp's query.  V rows whose
+// bit in (zm0, zm1) is clear (rows no query of the block can see: stale ring slots, the tail of the last page)
+// must not reach the output as 0 * (stale or non-finite).  Two ways, chosen by the caller:
+//   REG_MASK = false  zero those rows in the staged tile first (a pass over shared memory plus a proxy fence, but
+//                     only on tiles that have such rows: right for Full layers, where that is the last tile);
+//   REG_MASK = true   zero them in the A fragments after ldmatrix (four logic ops per fragment on every tile, no
+//                     pass over shared memory: right for rings, where most tiles have such rows).
+template <int D, bool REG_MASK = false>
 __device__ __forceinline__ void consume_tile(uint8_t* sV, uint32_t aK, uint32_t aV, uint32_t vm0, uint32_t vm1, bool wrote,
                                              const uint32_t (&qf)[D / 16][2], float scale_log2, float (&m_run)[2],
                                              float (&l_run)[2], float (&o)[D / 16][4], int lane, uint32_t zm0, uint32_t zm1) {
   constexpr int HALF_BYTES = TK * 128;
-  constexpr int CHUNKS = D / 8;
   constexpr int KS = D / 16;
   const int mi = lane >> 3, mr = lane & 7;
+  if constexpr (!REG_MASK) {
   if ((zm0 & zm1) != 0xffffffffu) {
-    // zero the V rows of invisible keys so that 0 * (stale or non-finite) cannot reach the output
+    constexpr int CHUNKS = D / 8;
     for (int idx = lane; idx < TK * CHUNKS; idx += 32) {
       const int row = idx / CHUNKS, ch = idx % CHUNKS;
       const bool v = ((row < 32 ? zm0 : zm1) >> (row & 31)) & 1u;
@@ -62,7 +67,8 @@ __device__ __forceinline__ void consume_tile(uint8_t* sV, uint32_t aK, uint32_t 
     }
     wrote = true;
   }
-  if (wrote) {
+  }
+  if (wrote) {  // this tile was patched through the generic proxy (zeroed rows, fused append)
     fence_proxy_async_smem();
     __syncwarp();
   }
@@ -126,18 +132,34 @@ __device__ __forceinline__ void consume_tile(uint8_t* sV, uint32_t aK, uint32_t 
       l_run[0] += f0.x + f1.x;  // sum the values the tensor core will actually multiply
       l_run[1] += f0.y + f1.y;
     }
-    // O^T += V^T P^T
+    // O^T += V^T P^T.  After the transposing load, a0 and a1 hold keys 16 kb + 2t, 2t + 1 (t = lane mod 4) in
+    // their halves, a2 and a3 hold keys 16 kb + 8 + 2t, 2t + 9.
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
       const uint32_t b0 = movmatrix_trans(pk[2 * kb]);
       const uint32_t b1 = movmatrix_trans(pk[2 * kb + 1]);
       const int key = kb * 16 + (mi >> 1) * 8 + mr;
+      if constexpr (!REG_MASK) {
 #pragma unroll
-      for (int mt = 0; mt < KS; ++mt) {
-        const int chunk = 2 * mt + (mi & 1);
-        uint32_t a0, a1, a2, a3;
-        ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
-        mma_bf16_16816(o[mt], a0, a1, a2, a3, b0, b1);
+        for (int mt = 0; mt < KS; ++mt) {
+          const int chunk = 2 * mt + (mi & 1);
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+          mma_bf16_16816(o[mt], a0, a1, a2, a3, b0, b1);
+        }
+      } else {
+        const uint32_t zw = kb < 2 ? zm0 : zm1;
+        const int sh = (kb & 1) * 16 + (lane & 3) * 2;
+        const uint32_t bits_lo = zw >> sh, bits_hi = zw >> (sh + 8);
+        const uint32_t keep_lo = ((bits_lo & 1u) ? 0x0000ffffu : 0u) | ((bits_lo & 2u) ? 0xffff0000u : 0u);
+        const uint32_t keep_hi = ((bits_hi & 1u) ? 0x0000ffffu : 0u) | ((bits_hi & 2u) ? 0xffff0000u : 0u);
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+          const int chunk = 2 * mt + (mi & 1);
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(aV + (chunk >> 3) * HALF_BYTES + swz128(key, chunk & 7), a0, a1, a2, a3);
+          mma_bf16_16816(o[mt], a0 & keep_lo, a1 & keep_lo, a2 & keep_hi, a3 & keep_hi, b0, b1);
+        }
       }
     }
   }
@@ -464,10 +486,10 @@ __global__ void __launch_bounds__(128, 2)
 decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p, const int n_items) {
   constexpr int NS = 3, NW = 3;
   constexpr int HALVES = D / 64;
-  constexpr int PPT = TK / P;
   constexpr int HALF_BYTES = TK * 128;
   constexpr int STAGE_BYTES = 2 * HALVES * HALF_BYTES;
-  constexpr int BOX_BYTES = P * 128;
+  constexpr int GR = P < HSWA_RING_GRANULE ? P : HSWA_RING_GRANULE;  // slots per TMA box
+  constexpr int NG = TK / GR;                                         // granules per tile
   constexpr int CHUNKS = D / 8;
   constexpr int KS = D / 16;
 
@@ -528,45 +550,42 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
           ok = false;
           break;
         }
-        uint32_t need = 0;
-        int pages[PPT];
-#pragma unroll
-        for (int i = 0; i < PPT; ++i) {
-          const int pgi = t * PPT + i;
-          pages[i] = __shfl_sync(0xffffffffu, pid, pgi & 31);
-          bool v = false;
-          if (pgi < M.R)
-            for (int s = lane; s < P; s += 32) v |= kr.valid(pgi * P + s);
-          if (__any_sync(0xffffffffu, v)) need |= 1u << i;
+        // The tile's TK slots are loaded in granules of GR slots (a granule never straddles a page), and only
+        // the granules that meet the window: the visible slots form the circular interval
+        // [head - min(W - 1, ctx), head].  Rows of granules that are not loaded keep whatever the stage buffer
+        // held; the consumers never let them count (masked scores, V fragments zeroed).
+        const int back = min(M.W - 1, kr.ctx);
+        const int start = math_mod(kr.head - back, M.C);
+        uint32_t okm = 0;
+        const int slot_lo = t * TK + (lane % NG) * GR;  // lane i < NG looks after granule i
+        const int pgi = slot_lo / P;
+        const int page_of = __shfl_sync(0xffffffffu, pid, pgi & 31);
+        if (lane < NG) {
+          if (pgi < M.R && (math_mod(slot_lo - start, M.C) <= back || math_mod(start - slot_lo, M.C) < GR)) {
+            if (page_of < 0 || page_of >= p.num_pages)
+              record_error(p.err, HSWA_ERR_BOUNDS, r, pgi, page_of);
+            else
+              okm = 1u << lane;
+          }
         }
+#pragma unroll
+        for (int sh = 1; sh < NG; sh <<= 1) okm |= __shfl_xor_sync(0xffffffffu, okm, sh);
+        const uint32_t full_bar = smem_u32(&bars[stage]);
         if (lane == 0) {
-          uint32_t okm = 0;
-#pragma unroll
-          for (int i = 0; i < PPT; ++i) {
-            if (!(need & (1u << i))) continue;
-            if (pages[i] < 0 || pages[i] >= p.num_pages) {
-              record_error(p.err, HSWA_ERR_BOUNDS, r, t * PPT + i, pages[i]);
-              continue;
-            }
-            okm |= 1u << i;
-          }
-          const uint32_t full_bar = smem_u32(&bars[stage]);
-          if (okm == 0) {
+          if (okm == 0)
             mbar_arrive(full_bar);
-          } else {
-            mbar_arrive_expect_tx(full_bar, __popc(okm) * 2 * HALVES * BOX_BYTES);
-            const uint32_t sb = smem_base + stage * STAGE_BYTES;
+          else
+            mbar_arrive_expect_tx(full_bar, __popc(okm) * 2 * HALVES * GR * 128);
+        }
+        __syncwarp();
+        if (lane < NG && (okm >> lane) & 1u) {
+          const uint32_t sb = smem_base + stage * STAGE_BYTES + lane * GR * 128;
+          const int slot_in_page = slot_lo % P;
 #pragma unroll
-            for (int i = 0; i < PPT; ++i) {
-              if (!(okm & (1u << i))) continue;
+          for (int kv = 0; kv < 2; ++kv)
 #pragma unroll
-              for (int kv = 0; kv < 2; ++kv)
-#pragma unroll
-                for (int hf = 0; hf < HALVES; ++hf)
-                  tma_load_4d(sb + (kv * HALVES + hf) * HALF_BYTES + i * BOX_BYTES, &tm_pool, full_bar, hf * 64, 0,
-                              kv * M.Hkv + kh, pages[i]);
-            }
-          }
+            for (int hf = 0; hf < HALVES; ++hf)
+              tma_load_4d(sb + (kv * HALVES + hf) * HALF_BYTES, &tm_pool, full_bar, hf * 64, slot_in_page, kv * M.Hkv + kh, page_of);
         }
         __syncwarp();
       }
@@ -576,23 +595,37 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     const int cw = warp - 1;
     const int g_row = lane >> 2;
     const int qd = (lane & 3) * 2;
-    griddep_wait();  // q, k_new, v_new and out may belong to the previous kernel on the stream
-    griddep_launch_dependents();
     int it = blockIdx.x;
     uint32_t qn[KS][2];
-    int ctx_n = 0, head_n = 0;
-    auto prefetch = [&](int item) {
-      const int r = item / M.Hkv, kh = item % M.Hkv;
+    int ctx_n = 0, head_n = 0, pid_n = -1;
+    // fused append: the new token's K (lanes [0, CHUNKS)) and V (lanes [CHUNKS, 2 CHUNKS)) row of the next ring, one
+    // 16-byte chunk per lane, fetched one ring ahead like Q
+    static_assert(2 * CHUNKS <= 32, "one chunk of the new K/V row per lane");
+    uint4 an = make_uint4(0, 0, 0, 0);
+    // lengths, ring head and ring table do not change during a step: they may be read before the previous
+    // kernel on the stream has finished (lane i keeps page id i of the ring)
+    auto prefetch_meta = [&](int item) {
+      const int r = item / M.Hkv;
       ctx_n = p.b.ctx_len[r];
       head_n = p.b.ring_head[r];
+      pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
+    };
+    auto prefetch_qkv = [&](int item) {
+      const int r = item / M.Hkv, kh = item % M.Hkv;
       const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
         qn[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
         qn[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
       }
+      if (fuse && lane < 2 * CHUNKS)
+        an = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D +
+                                             (lane % CHUNKS) * 8);
     };
-    if (it < n_items) prefetch(it);
+    if (it < n_items) prefetch_meta(it);
+    griddep_wait();  // q, k_new, v_new and out may belong to the previous kernel on the stream
+    griddep_launch_dependents();
+    if (it < n_items) prefetch_qkv(it);
     for (int k = 0; it < n_items; ++k, it += gridDim.x) {
       const int r = it / M.Hkv, kh = it % M.Hkv;
       uint32_t qf[KS][2];
@@ -609,7 +642,12 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       kr.W = M.W;
       kr.C = M.C;
       const int ctx = ctx_n;
-      if (it + gridDim.x < n_items) prefetch(it + gridDim.x);
+      const uint4 a_cur = an;
+      const int pid_cur = pid_n;
+      if (it + gridDim.x < n_items) {
+        prefetch_meta(it + gridDim.x);
+        prefetch_qkv(it + gridDim.x);
+      }
 
       float m_run[2] = {-INFINITY, -INFINITY};
       float l_run[2] = {0.f, 0.f};
@@ -633,23 +671,21 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         if (fuse && kr.head >= tile_lo && kr.head < tile_lo + TK) {
           // fused append: the new token goes to ring slot ring_head, in the staged tile and in the cache
           const int row = kr.head - tile_lo;
-          const int page = p.b.ring_table[(int64_t)r * M.R + kr.head / P];
+          const int page = __shfl_sync(0xffffffffu, pid_cur, kr.head / P);
           const int slot = kr.head % P;
           const bool page_ok = page >= 0 && page < p.num_pages;
           if (!page_ok && lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, page);
-          for (int c = lane; c < 2 * CHUNKS; c += 32) {
-            const int kv = c / CHUNKS, ch = c % CHUNKS;
-            const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D + ch * 8;
-            const uint4 val = *reinterpret_cast<const uint4*>(src);
-            *reinterpret_cast<uint4*>((kv == 0 ? sK : sV) + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = val;
+          if (lane < 2 * CHUNKS) {
+            const int kv = lane / CHUNKS, ch = lane % CHUNKS;
+            *reinterpret_cast<uint4*>((kv == 0 ? sK : sV) + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = a_cur;
             if (page_ok)
-              *reinterpret_cast<uint4*>(p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * P + slot) * D + ch * 8) = val;
+              *reinterpret_cast<uint4*>(p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * P + slot) * D + ch * 8) = a_cur;
           }
           wrote = true;
         }
         const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
         const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
-        consume_tile<D>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
+        consume_tile<D, true>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
       }
@@ -676,26 +712,32 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         sc_ml[(cw * 8 + qd + 1) * 2 + 1] = l_run[1];
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");
-      for (int idx = threadIdx.x - 32; idx < M.G * D; idx += NW * 32) {
-        const int g = idx / D, d = idx % D;
+      for (int idx = threadIdx.x - 32; idx < M.G * (D / 4); idx += NW * 32) {
+        const int g = idx / (D / 4), d = (idx % (D / 4)) * 4;
         float mm = -INFINITY;
 #pragma unroll
         for (int w = 0; w < NW; ++w) mm = fmaxf(mm, sc_ml[(w * 8 + g) * 2]);
-        float L = 0.f, O = 0.f;
+        float L = 0.f;
+        float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
         if (mm != -INFINITY) {
 #pragma unroll
           for (int w = 0; w < NW; ++w) {
             const float f = fast_exp2(sc_ml[(w * 8 + g) * 2] - mm);
+            const float4 x = *reinterpret_cast<const float4*>(&sc_o[(w * 8 + g) * D + d]);
             L += f * sc_ml[(w * 8 + g) * 2 + 1];
-            O += f * sc_o[(w * 8 + g) * D + d];
+            O.x += f * x.x;
+            O.y += f * x.y;
+            O.z += f * x.z;
+            O.w += f * x.w;
           }
         }
         const int64_t row = (int64_t)r * M.Hq + kh * M.G + g;
-        const float val = L > 0.f ? O / L : 0.f;
+        const float inv = L > 0.f ? 1.f / L : 0.f;
         if (M.out_fp32)
-          reinterpret_cast<float*>(p.out)[row * D + d] = val;
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + row * D + d) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
         else
-          reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d] = __float2bfloat16_rn(val);
+          *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.out) + row * D + d) =
+              make_uint2(pack_bf16x2(O.x * inv, O.y * inv), pack_bf16x2(O.z * inv, O.w * inv));
         if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");  // scratch may be rewritten

@@ -106,6 +106,8 @@ struct PrefillParams {
 
 // Launchers implemented in the kernel translation units.
 cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s);
+// Slots per TMA box of the persistent ring decode kernel (its tensor map is built with this box height).
+#define HSWA_RING_GRANULE 16
 cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
                                cudaStream_t s);
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);

@@ -96,6 +96,27 @@ def test_decode_config1(is_swa, fused):
     assert err <= TOL and lerr <= TOL, (err, lerr)
 
 
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(4, 64, 16, 1)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_decode_ignores_nonfinite_stale_slots(d, is_swa):
+    """Slots that hold no valid token (stale ring slots, page tails, unused pages) are filled with +inf (K) and
+    NaN (V) instead of the finite poison: decode must neither read them into a score that counts nor let
+    0 * NaN reach the output (Sec. 3.1.3: reading an invalid slot degrades correctness)."""
+    from helpers import POISON_K, POISON_V
+    W, C = d.window, d.ring_slots
+    ctx = [0, 1, 5, 63, 64, 100, W - 1, W, W + 1, C, C + 7, 1000, 2049]
+    sc = build_scenario(d, ctx, [1] * len(ctx), seed=91)
+    pk, pv = wl.bf16_bits_const(POISON_K, (1,))[0], wl.bf16_bits_const(POISON_V, (1,))[0]
+    for pool in (sc.full_pool, sc.swa_pool):
+        n_k, n_v = int((pool[:, 0] == pk).sum()), int((pool[:, 1] == pv).sum())
+        assert n_k > 0 and n_v > 0
+        pool[:, 0][pool[:, 0] == pk] = 0x7F80  # +inf
+        pool[:, 1][pool[:, 1] == pv] = 0x7FC0  # NaN
+    for fused in (True, False):
+        err, lerr = run_decode(sc, is_swa, fused)
+        assert err <= TOL and lerr <= TOL, (fused, err, lerr)
+
+
 @pytest.mark.parametrize("d", [dims(4, 64, 16, 1), dims(8, 128, 64), dims(1, 128, 64, 3), dims(3, 64, 32),
                                dims(8, 128, 16), dims(5, 64, 64)], ids=str)
 @pytest.mark.parametrize("is_swa", [False, True])
