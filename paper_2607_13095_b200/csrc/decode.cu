@@ -796,7 +796,7 @@ struct KeyRangeMulti {
   }
 };
 
-template <int D, int P, int NS>
+template <int D, int P, int NS, bool SWA>  // SWA: rings, where most tiles hold stale slots (V masked in registers)
 __global__ void __launch_bounds__(160, 2)
 decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
   constexpr int HALVES = D / 64;
@@ -946,7 +946,7 @@ decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParam
       const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane, w));
       const uint32_t zm0 = __ballot_sync(0xffffffffu, kr.any(tile_lo + lane));
       const uint32_t zm1 = __ballot_sync(0xffffffffu, kr.any(tile_lo + 32 + lane));
-      consume_tile<D>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, zm0, zm1);
+      consume_tile<D, SWA>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, zm0, zm1);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
     }
@@ -1000,7 +1000,7 @@ cudaError_t launch_mtp_t(const CUtensorMap& tm, const DecodeParams& p, cudaStrea
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
   constexpr int SMEM = NS * STAGE_BYTES + 1024;
   static_assert(4 * 8 * D * 4 + 4 * 64 <= NS * STAGE_BYTES, "per-token results must fit the stage buffers");
-  auto kern = decode_mtp_kernel<D, P, NS>;
+  auto kern = p.is_swa ? decode_mtp_kernel<D, P, NS, true> : decode_mtp_kernel<D, P, NS, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   dim3 grid(p.b.B, p.grid_splits, p.m.Hkv);
