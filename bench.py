@@ -34,7 +34,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep", "prefetch"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep", "prefetch", "buckets"])
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
@@ -388,6 +388,49 @@ def run_prefix_sweep(args, torch, device, peaks):
                               "about 0.12x at a 1M prefix (unnamed GPU), attention alone falls further"}))
 
 
+def run_length_buckets(args, torch, device):
+    """Paper Sec. 5.3 (length bucketing): when requests whose cached prefixes differ a lot are scheduled into the
+    same chunked-prefill step of one instance, its data-parallel attention ranks synchronise after every layer and
+    all wait for the rank with the longest prefix.  Emulates one instance of 8 such ranks on this GPU, one rank at
+    a time: a rank's work is one request's 16K-token chunk over its cached prefix through one hybrid block
+    (1 Full + 6 SWA layers), and a synchronised step costs its slowest rank.  48 seeded requests (24 / 16 / 8 in
+    the paper's tiers 0-64K / 64K-256K / 256K-1M) are scheduled in arrival order and with the three-tier bucketing
+    (every step's 8 requests come from one tier); the balanced bound is the sum of all times / 8."""
+    from paper_2607_13095_b200 import workloads as wl
+    chunk, ranks = args.chunk or 16384, 8
+    rng = np.random.default_rng(53)
+    tiers = [(0, 65536, 24), (65536, 262144, 16), (262144, 1048576 - chunk, 8)]
+    reqs = [(ti, int(rng.integers(lo, hi))) for ti, (lo, hi, n) in enumerate(tiers) for _ in range(n)]
+    order = rng.permutation(len(reqs))  # arrival order
+    ms = []
+    for ti, prefix in reqs:
+        t = wl.make_tables(wl.BIG, [prefix], [chunk], seed=7, slack=1.0)
+        w = wl.Workload(f"prefix{prefix}-chunk{chunk}", wl.BIG, wl.hybrid_layer_flags(7)[:2], t, 7)
+        pb = PrefillBench(w, device)
+        ms_full = time_events(torch, lambda: pb.run_layer(0), 1, 1 if prefix > 262144 else 2)
+        ms_swa = time_events(torch, lambda: pb.run_layer(1), 1, 3)
+        ms.append(ms_full + 6 * ms_swa)
+        del pb
+        torch.cuda.empty_cache()
+    ms = np.array(ms)
+
+    def schedule(seq):
+        return float(sum(ms[seq[i:i + ranks]].max() for i in range(0, len(seq), ranks)))
+
+    arrival = [int(i) for i in order]
+    bucketed = sorted(arrival, key=lambda i: reqs[i][0])  # stable: arrival order inside a tier
+    t_mixed, t_bucket, t_bound = schedule(arrival), schedule(bucketed), float(ms.sum() / ranks)
+    tokens = len(reqs) * chunk
+    print(json.dumps({
+        "metric": "prefill_attn_tokens_per_s_bucketed_vs_arrival_order", "unit": "x", "value": t_mixed / t_bucket,
+        "chunk": chunk, "ranks": ranks, "requests": len(reqs), "n_gpus": 1, "data": "synthetic", "dtype": "bf16",
+        "tokens_per_s": {"arrival_order": tokens / (t_mixed * 1e-3), "three_tier_buckets": tokens / (t_bucket * 1e-3),
+                         "balanced_bound": tokens / (t_bound * 1e-3)},
+        "block_ms_by_tier": [float(ms[[i for i, r_ in enumerate(reqs) if r_[0] == ti]].mean()) for ti in range(3)],
+        "note": "8 data-parallel attention ranks of one instance emulated one at a time on one GPU; a step costs its "
+                "slowest rank (per-layer synchronisation before the MoE stage); attention + append of one hybrid block"}))
+
+
 def run_layerwise_prefetch(args, torch, device):
     """Paper Sec. 3.1.2 (layerwise KVCache prefetch): the SWA state of every request lives in pinned host memory
     (W - 1 tokens per request and SWA layer: the only part a resumed request needs) and is loaded back layer by
@@ -553,6 +596,9 @@ def main():
         return
     if args.workload == "prefix_sweep":
         run_prefix_sweep(args, torch, device, peaks)
+        return
+    if args.workload == "buckets":
+        run_length_buckets(args, torch, device)
         return
     if args.workload == "cfg3":
         run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks)
