@@ -397,9 +397,10 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + o_bytes);
   }
   CUtensorMap tm;
-  if ((st = make_pool_map(h, layer, &tm)) != HSWA_OK) return st;
+  const int granule = h->cfg.page_size < HSWA_RING_GRANULE ? h->cfg.page_size : HSWA_RING_GRANULE;
+  if ((st = make_pool_map(h, layer, &tm, layer->is_swa ? granule : 0)) != HSWA_OK) return st;
   if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
-  if (hswa_launch_decode_mtp(tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (hswa_launch_decode_mtp(h, tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   return HSWA_OK;
 }

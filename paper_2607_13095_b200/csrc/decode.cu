@@ -503,7 +503,12 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const ModelParams& M = p.m;
   const int n_tiles = (M.C + TK - 1) / TK;
-  const bool fuse = p.k_new != nullptr;
+  const bool fuse = p.k_new != nullptr;  // one new token per request, appended here (nq == 1 only)
+  // With nq > 1 (a decode step that carries draft tokens, already appended by the caller) a work item is one
+  // token of one ring: token w of a request sits at position ctx + w in slot ring_head + w, so it sees the ring
+  // exactly as a single new token of a request with ctx + w cached tokens and that ring head would (later
+  // drafts lie ahead of its slot, more than W - 1 slots "back" around the ring, because nq <= C - W + 1).
+  const int nq = p.nq;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -520,14 +525,14 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     int it = blockIdx.x;
     int ctx_n = 0, head_n = 0, pid_n = 0;
     if (it < n_items) {
-      const int r = it / M.Hkv;
-      ctx_n = p.b.ctx_len[r];
-      head_n = p.b.ring_head[r];
+      const int r = it / (M.Hkv * nq), w = it % nq;
+      ctx_n = p.b.ctx_len[r] + w;
+      head_n = math_mod(p.b.ring_head[r] + w, M.C);
       pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : 0;
     }
     bool ok = true;
     for (int k = 0; it < n_items && ok; ++k, it += gridDim.x) {
-      const int r = it / M.Hkv, kh = it % M.Hkv;
+      const int r = it / (M.Hkv * nq), kh = (it / nq) % M.Hkv;
       KeyRange kr;
       kr.is_swa = 1;
       kr.span = M.C;
@@ -538,9 +543,9 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       const int pid = pid_n;
       const int nxt = it + gridDim.x;
       if (nxt < n_items) {  // next ring's metadata, one ring ahead of its first TMA
-        const int rn = nxt / M.Hkv;
-        ctx_n = p.b.ctx_len[rn];
-        head_n = p.b.ring_head[rn];
+        const int rn = nxt / (M.Hkv * nq), wn = nxt % nq;
+        ctx_n = p.b.ctx_len[rn] + wn;
+        head_n = math_mod(p.b.ring_head[rn] + wn, M.C);
         pid_n = lane < M.R ? p.b.ring_table[(int64_t)rn * M.R + lane] : 0;
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
@@ -605,14 +610,14 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     // lengths, ring head and ring table do not change during a step: they may be read before the previous
     // kernel on the stream has finished (lane i keeps page id i of the ring)
     auto prefetch_meta = [&](int item) {
-      const int r = item / M.Hkv;
-      ctx_n = p.b.ctx_len[r];
-      head_n = p.b.ring_head[r];
+      const int r = item / (M.Hkv * nq), w = item % nq;
+      ctx_n = p.b.ctx_len[r] + w;
+      head_n = math_mod(p.b.ring_head[r] + w, M.C);
       pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
     };
     auto prefetch_qkv = [&](int item) {
-      const int r = item / M.Hkv, kh = item % M.Hkv;
-      const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
+      const int r = item / (M.Hkv * nq), kh = (item / nq) % M.Hkv, w = item % nq;
+      const __nv_bfloat16* qrow = p.q + (((int64_t)r * nq + w) * M.Hq + kh * M.G + g_row) * D;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
         qn[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
@@ -627,7 +632,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     griddep_launch_dependents();
     if (it < n_items) prefetch_qkv(it);
     for (int k = 0; it < n_items; ++k, it += gridDim.x) {
-      const int r = it / M.Hkv, kh = it % M.Hkv;
+      const int r = it / (M.Hkv * nq), kh = (it / nq) % M.Hkv, w_tok = it % nq;
       uint32_t qf[KS][2];
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -731,7 +736,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
             O.w += f * x.w;
           }
         }
-        const int64_t row = (int64_t)r * M.Hq + kh * M.G + g;
+        const int64_t row = ((int64_t)r * nq + w_tok) * M.Hq + kh * M.G + g;
         const float inv = L > 0.f ? 1.f / L : 0.f;
         if (M.out_fp32)
           *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + row * D + d) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
@@ -752,7 +757,7 @@ cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const Dec
   auto kern = decode_ring_kernel<D, P>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
-  const int n_items = p.b.B * p.m.Hkv;
+  const int n_items = p.b.B * p.m.Hkv * p.nq;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_items < 2 * h->num_sms ? n_items : 2 * h->num_sms, 1, 1);
   cfg.blockDim = dim3(128, 1, 1);
@@ -768,35 +773,22 @@ cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const Dec
 
 
 // ---------------------------------------------------------------------------------------------------------
-// Multi-token decode (paper Sec. 6.2: the model drafts with 3 MTP layers, so a decode step carries the last
-// accepted token plus up to 3 drafts per request).  The nq new tokens are already in the cache (the append
-// runs first on the stream: on a ring that is safe for nq <= C - W + 1).  One consumer warp per draft token:
-// every warp walks every staged tile with its own Q, its own causal / window mask and its own softmax state,
-// so the KV bytes are streamed once for all nq tokens and no cross-warp merge is needed.
+// Multi-token decode on Full layers (paper Sec. 6.2: the model drafts with 3 MTP layers, so a decode step
+// carries the last accepted token plus up to 3 drafts per request).  The nq new tokens are already in the cache
+// (the append runs first on the stream).  One consumer warp per draft token: every warp walks every staged tile
+// with its own Q, its own causal mask and its own softmax state, so the KV bytes are streamed from HBM once for
+// all nq tokens and no cross-warp merge is needed.  (Two tokens per warp sharing the K / V fragments was
+// measured: same time, so shared-memory traffic is not what bounds this kernel.)  On SWA layers a multi-token
+// step runs through the ring kernel, one work item per ring and token.
 struct KeyRangeMulti {
-  int is_swa, span, k_begin, head, ctx, W, C, nq;
-  __device__ __forceinline__ int slot_pos(int idx) const {  // position held by ring slot idx after the append
-    int off = idx - head;
-    if (off < 0) off += C;
-    return off < nq ? ctx + off : ctx + off - C;
-  }
-  // visible to draft token w (absolute position ctx + w)?
-  __device__ __forceinline__ bool valid(int idx, int w) const {
-    if (!is_swa) return idx < span && k_begin + idx <= ctx + w;
-    if (idx >= C) return false;
-    const int pos = slot_pos(idx);
-    return pos >= 0 && pos <= ctx + w && pos > ctx + w - W;
-  }
+  int span, k_begin, ctx;
+  // key idx of this split visible to draft token w (absolute position ctx + w)?
+  __device__ __forceinline__ bool valid(int idx, int w) const { return idx < span && k_begin + idx <= ctx + w; }
   // visible to at least one of the nq tokens?
-  __device__ __forceinline__ bool any(int idx) const {
-    if (!is_swa) return idx < span;
-    if (idx >= C) return false;
-    const int pos = slot_pos(idx);
-    return pos >= 0 && pos <= ctx + nq - 1 && pos > ctx - W;
-  }
+  __device__ __forceinline__ bool any(int idx) const { return idx < span; }
 };
 
-template <int D, int P, int NS, bool SWA>  // SWA: rings, where most tiles hold stale slots (V masked in registers)
+template <int D, int P, int NS>
 __global__ void __launch_bounds__(160, 2)
 decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
   constexpr int HALVES = D / 64;
@@ -819,22 +811,10 @@ decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParam
   const int kv_len = ctx + nq;
 
   KeyRangeMulti kr;
-  kr.is_swa = p.is_swa;
   kr.ctx = ctx;
-  kr.W = M.W;
-  kr.C = M.C;
-  kr.nq = nq;
-  kr.head = 0;
-  kr.k_begin = 0;
-  if (!p.is_swa) {
-    kr.k_begin = split * p.split_len;
-    if (kr.k_begin >= kv_len) return;
-    kr.span = min(kv_len, kr.k_begin + p.split_len) - kr.k_begin;
-  } else {
-    if (split > 0) return;
-    kr.head = p.b.ring_head[r];
-    kr.span = M.C;
-  }
+  kr.k_begin = split * p.split_len;
+  if (kr.k_begin >= kv_len) return;
+  kr.span = min(kv_len, kr.k_begin + p.split_len) - kr.k_begin;
   const int n_tiles = (kr.span + TK - 1) / TK;
 
   if (threadIdx.x == 0) {
@@ -855,15 +835,8 @@ decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParam
   const int qd = (lane & 3) * 2;
 
   if (warp == 0) {
-    const int32_t* tbl;
-    int n_pages;
-    if (!p.is_swa) {
-      tbl = p.b.block_table + (int64_t)r * p.b.max_blocks + kr.k_begin / P;
-      n_pages = (kr.span + P - 1) / P;
-    } else {
-      tbl = p.b.ring_table + (int64_t)r * M.R;
-      n_pages = M.R;
-    }
+    const int32_t* tbl = p.b.block_table + (int64_t)r * p.b.max_blocks + kr.k_begin / P;
+    const int n_pages = (kr.span + P - 1) / P;
     int pid_next = lane < n_pages ? tbl[lane] : 0;
     int pid_cur = 0;
     for (int t = 0; t < n_tiles; ++t) {
@@ -946,7 +919,7 @@ decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParam
       const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane, w));
       const uint32_t zm0 = __ballot_sync(0xffffffffu, kr.any(tile_lo + lane));
       const uint32_t zm1 = __ballot_sync(0xffffffffu, kr.any(tile_lo + 32 + lane));
-      consume_tile<D, SWA>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, zm0, zm1);
+      consume_tile<D>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, zm0, zm1);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
     }
@@ -1000,7 +973,7 @@ cudaError_t launch_mtp_t(const CUtensorMap& tm, const DecodeParams& p, cudaStrea
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
   constexpr int SMEM = NS * STAGE_BYTES + 1024;
   static_assert(4 * 8 * D * 4 + 4 * 64 <= NS * STAGE_BYTES, "per-token results must fit the stage buffers");
-  auto kern = p.is_swa ? decode_mtp_kernel<D, P, NS, true> : decode_mtp_kernel<D, P, NS, false>;
+  auto kern = decode_mtp_kernel<D, P, NS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   dim3 grid(p.b.B, p.grid_splits, p.m.Hkv);
@@ -1064,9 +1037,10 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t hswa_launch_decode_mtp(const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
+cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
   if (p.nq < 1 || p.nq > 4) return cudaErrorInvalidValue;
+  if (p.is_swa) return hswa_launch_decode(h, tm_pool, p, false, s);  // rings: one work item per (ring, token)
   const int D = p.m.D, P = p.m.P;
   if (D == 128 && P == 64) return launch_mtp_t<128, 64, 3>(tm_pool, p, s);
   if (D == 128 && P == 32) return launch_mtp_t<128, 32, 3>(tm_pool, p, s);
