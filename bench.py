@@ -749,6 +749,21 @@ def main():
         "roofline": roofline, "clocks": clocks.summary(), "e2e": e2e,
         "gpu_launches": bench.launches_per_step * args.steps,
     }
+    if not args.no_graph and world == 1:
+        # The same device-resident step replayed as one CUDA graph (reported separately: the host's launch time
+        # matters at small batch, where a layer's kernels are shorter than the calls that launch them).
+        try:
+            bench.reset()
+            bench.step()
+            torch.cuda.synchronize()
+            g_step = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_step):
+                bench.step()
+            n_rep = min(args.steps, 2 * total_steps + 4)
+            line["step_as_cuda_graph_ms"] = time_events(torch, g_step.replay, 3, max(1, n_rep - 3))
+        except Exception as ex:  # noqa: BLE001
+            sys.stderr.write(f"bench: step graph capture failed ({ex})\n")
+            torch.cuda.synchronize()
     if not args.no_cpu_baseline and world == 1:
         bench.reset()
         line["cpu_baseline"] = cpu_baseline_decode(bench)
