@@ -549,7 +549,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
           const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));
           v[k] = pack_bf16x2(e.x, e.y);
           // the row sum takes the fp32 values before their rounding to bf16 (summing the rounded ones instead
-          // costs one more ALU op per key and 6.5 % of the kernel's time; the difference shows only for nearly
+          // costs one more ALU op per key and 7-8 % of the kernel's time; the difference shows only for nearly
           // one-hot rows, where it is bounded by 2^-9 max|v|)
           acc[k & 3] = __fadd2_rn(acc[k & 3], e);
           if (part > 0 && (part % QPP) == 0 && k == part * 16 + 7) {
@@ -1080,7 +1080,7 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));  // masked columns: 2^(-inf) = 0
           v[k] = pack_bf16x2(e.x, e.y);
           // the row sum takes the fp32 values before their rounding to bf16 (summing the rounded ones instead
-          // costs one more ALU op per key and 6.5 % of the kernel's time; the difference shows only for nearly
+          // costs one more ALU op per key and 7-8 % of the kernel's time; the difference shows only for nearly
           // one-hot rows, where it is bounded by 2^-9 max|v|)
           acc[k & 3] = __fadd2_rn(acc[k & 3], e);
         }
