@@ -341,6 +341,8 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   if (q_len == 1) return decode_impl(h, layer, b, 0, q, k_new, v_new, out, lse, workspace, workspace_bytes, stream);
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
+  // a ring kernel with the append fused may start early behind another fused decode kernel of the same step
+  const bool early = layer->is_swa && h->chain_ok && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len;
   h->chain_ok = 0;
   if (b->q_indptr != nullptr || q_len < 1 || q_len > 4) return HSWA_ERR_INVALID_ARG;
   if (b->batch == 0) return HSWA_OK;
@@ -367,8 +369,10 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   p.num_pages = a.num_pages;
   p.is_swa = layer->is_swa;
   p.q = static_cast<const __nv_bfloat16*>(q);
-  p.k_new = nullptr;  // the tokens are in the cache by the time the attention kernel runs
-  p.v_new = nullptr;
+  // Full layers: the tokens are in the cache by the time the attention kernel runs (append kernel first); rings:
+  // the ring kernel appends them itself
+  p.k_new = layer->is_swa ? a.k_new : nullptr;
+  p.v_new = layer->is_swa ? a.v_new : nullptr;
   p.out = out;
   p.lse = lse;
   p.err = h->err;
@@ -399,9 +403,12 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   CUtensorMap tm;
   const int granule = h->cfg.page_size < HSWA_RING_GRANULE ? h->cfg.page_size : HSWA_RING_GRANULE;
   if ((st = make_pool_map(h, layer, &tm, layer->is_swa ? granule : 0)) != HSWA_OK) return st;
-  if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
-  if (hswa_launch_decode_mtp(h, tm, p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (!layer->is_swa && hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (hswa_launch_decode_mtp(h, tm, p, early, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  h->chain_ok = 1;  // none of these kernels writes the batch arrays or another layer's pool
+  h->chain_stream = stream;
+  h->chain_ctx = (const void*)b->ctx_len;
   return HSWA_OK;
 }
 

@@ -503,11 +503,13 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const ModelParams& M = p.m;
   const int n_tiles = (M.C + TK - 1) / TK;
-  const bool fuse = p.k_new != nullptr;  // one new token per request, appended here (nq == 1 only)
-  // With nq > 1 (a decode step that carries draft tokens, already appended by the caller) a work item is one
-  // token of one ring: token w of a request sits at position ctx + w in slot ring_head + w, so it sees the ring
-  // exactly as a single new token of a request with ctx + w cached tokens and that ring head would (later
-  // drafts lie ahead of its slot, more than W - 1 slots "back" around the ring, because nq <= C - W + 1).
+  const bool fuse = p.k_new != nullptr;  // the new tokens are appended here; otherwise they are in the cache already
+  // With nq > 1 (a decode step that carries draft tokens) the ring's tiles are staged once and walked once per
+  // token: token w of a request sits at position ctx + w in slot ring_head + w, so it sees the ring exactly as a
+  // single new token of a request with ctx + w cached tokens and that ring head would (later drafts lie ahead of
+  // its slot, more than W - 1 slots "back" around the ring, because nq <= C - W + 1).  When the append is fused,
+  // the pass of token w patches row w into the staged tile (rows 0 .. w - 1 are there from the earlier passes)
+  // and writes it to the cache.
   const int nq = p.nq;
 
   if (threadIdx.x == 0) {
@@ -525,14 +527,14 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     int it = blockIdx.x;
     int ctx_n = 0, head_n = 0, pid_n = 0;
     if (it < n_items) {
-      const int r = it / (M.Hkv * nq), w = it % nq;
-      ctx_n = p.b.ctx_len[r] + w;
-      head_n = math_mod(p.b.ring_head[r] + w, M.C);
+      const int r = it / M.Hkv;
+      ctx_n = p.b.ctx_len[r];
+      head_n = p.b.ring_head[r];
       pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : 0;
     }
     bool ok = true;
     for (int k = 0; it < n_items && ok; ++k, it += gridDim.x) {
-      const int r = it / (M.Hkv * nq), kh = (it / nq) % M.Hkv;
+      const int r = it / M.Hkv, kh = it % M.Hkv;
       KeyRange kr;
       kr.is_swa = 1;
       kr.span = M.C;
@@ -543,9 +545,9 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       const int pid = pid_n;
       const int nxt = it + gridDim.x;
       if (nxt < n_items) {  // next ring's metadata, one ring ahead of its first TMA
-        const int rn = nxt / (M.Hkv * nq), wn = nxt % nq;
-        ctx_n = p.b.ctx_len[rn] + wn;
-        head_n = math_mod(p.b.ring_head[rn] + wn, M.C);
+        const int rn = nxt / M.Hkv;
+        ctx_n = p.b.ctx_len[rn];
+        head_n = p.b.ring_head[rn];
         pid_n = lane < M.R ? p.b.ring_table[(int64_t)rn * M.R + lane] : 0;
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
@@ -556,17 +558,18 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
           break;
         }
         // The tile's TK slots are loaded in granules of GR slots (a granule never straddles a page), and only
-        // the granules that meet the window: the visible slots form the circular interval
-        // [head - min(W - 1, ctx), head].  Rows of granules that are not loaded keep whatever the stage buffer
-        // held; the consumers never let them count (masked scores, V fragments zeroed).
+        // the granules that meet the window: the slots visible to at least one of the nq tokens form the circular
+        // interval [head - min(W - 1, ctx), head + nq - 1].  Rows of granules that are not loaded keep whatever the
+        // stage buffer held; the consumers never let them count (masked scores, V fragments zeroed).
         const int back = min(M.W - 1, kr.ctx);
         const int start = math_mod(kr.head - back, M.C);
+        const int last = back + nq - 1;  // offset of the last visible slot from `start`
         uint32_t okm = 0;
         const int slot_lo = t * TK + (lane % NG) * GR;  // lane i < NG looks after granule i
         const int pgi = slot_lo / P;
         const int page_of = __shfl_sync(0xffffffffu, pid, pgi & 31);
         if (lane < NG) {
-          if (pgi < M.R && (math_mod(slot_lo - start, M.C) <= back || math_mod(start - slot_lo, M.C) < GR)) {
+          if (pgi < M.R && (math_mod(slot_lo - start, M.C) <= last || math_mod(start - slot_lo, M.C) < GR)) {
             if (page_of < 0 || page_of >= p.num_pages)
               record_error(p.err, HSWA_ERR_BOUNDS, r, pgi, page_of);
             else
@@ -603,20 +606,20 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     int it = blockIdx.x;
     uint32_t qn[KS][2];
     int ctx_n = 0, head_n = 0, pid_n = -1;
-    // fused append: the new token's K (lanes [0, CHUNKS)) and V (lanes [CHUNKS, 2 CHUNKS)) row of the next ring, one
-    // 16-byte chunk per lane, fetched one ring ahead like Q
+    // fused append: the K (lanes [0, CHUNKS)) and V (lanes [CHUNKS, 2 CHUNKS)) row of the next token, one 16-byte
+    // chunk per lane, fetched one pass ahead like Q
     static_assert(2 * CHUNKS <= 32, "one chunk of the new K/V row per lane");
     uint4 an = make_uint4(0, 0, 0, 0);
     // lengths, ring head and ring table do not change during a step: they may be read before the previous
     // kernel on the stream has finished (lane i keeps page id i of the ring)
     auto prefetch_meta = [&](int item) {
-      const int r = item / (M.Hkv * nq), w = item % nq;
-      ctx_n = p.b.ctx_len[r] + w;
-      head_n = math_mod(p.b.ring_head[r] + w, M.C);
+      const int r = item / M.Hkv;
+      ctx_n = p.b.ctx_len[r];
+      head_n = p.b.ring_head[r];
       pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
     };
-    auto prefetch_qkv = [&](int item) {
-      const int r = item / (M.Hkv * nq), kh = (item / nq) % M.Hkv, w = item % nq;
+    auto prefetch_qkv = [&](int item, int w) {
+      const int r = item / M.Hkv, kh = item % M.Hkv;
       const __nv_bfloat16* qrow = p.q + (((int64_t)r * nq + w) * M.Hq + kh * M.G + g_row) * D;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -624,15 +627,18 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         qn[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
       }
       if (fuse && lane < 2 * CHUNKS)
-        an = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D +
+        an = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) + (((int64_t)r * nq + w) * M.Hkv + kh) * D +
                                              (lane % CHUNKS) * 8);
     };
     if (it < n_items) prefetch_meta(it);
     griddep_wait();  // q, k_new, v_new and out may belong to the previous kernel on the stream
     griddep_launch_dependents();
-    if (it < n_items) prefetch_qkv(it);
+    if (it < n_items) prefetch_qkv(it, 0);
     for (int k = 0; it < n_items; ++k, it += gridDim.x) {
-      const int r = it / (M.Hkv * nq), kh = (it / nq) % M.Hkv, w_tok = it % nq;
+      const int r = it / M.Hkv, kh = it % M.Hkv;
+      const int ctx0 = ctx_n, head0 = head_n, pid_cur = pid_n;
+      if (it + gridDim.x < n_items) prefetch_meta(it + gridDim.x);
+     for (int w_tok = 0; w_tok < nq; ++w_tok) {
       uint32_t qf[KS][2];
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -642,17 +648,16 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       KeyRange kr;
       kr.is_swa = 1;
       kr.span = M.C;
-      kr.head = head_n;
-      kr.ctx = ctx_n;
+      kr.head = math_mod(head0 + w_tok, M.C);
+      kr.ctx = ctx0 + w_tok;
       kr.W = M.W;
       kr.C = M.C;
-      const int ctx = ctx_n;
+      const int ctx = kr.ctx;
       const uint4 a_cur = an;
-      const int pid_cur = pid_n;
-      if (it + gridDim.x < n_items) {
-        prefetch_meta(it + gridDim.x);
-        prefetch_qkv(it + gridDim.x);
-      }
+      if (w_tok + 1 < nq)
+        prefetch_qkv(it, w_tok + 1);
+      else if (it + gridDim.x < n_items)
+        prefetch_qkv(it + gridDim.x, 0);
 
       float m_run[2] = {-INFINITY, -INFINITY};
       float l_run[2] = {0.f, 0.f};
@@ -662,7 +667,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       bool ok = true;
       for (int t = cw; t < n_tiles; t += NW) {
         const int g = k * n_tiles + t, stage = g % NS;
-        if (!mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {
+        if (w_tok == 0 && !mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {  // later passes reuse the staged tile
           if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
           ok = false;
           break;
@@ -674,7 +679,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         const int tile_lo = t * TK;
         bool wrote = false;
         if (fuse && kr.head >= tile_lo && kr.head < tile_lo + TK) {
-          // fused append: the new token goes to ring slot ring_head, in the staged tile and in the cache
+          // fused append: this pass's token goes to its ring slot, in the staged tile and in the cache
           const int row = kr.head - tile_lo;
           const int page = __shfl_sync(0xffffffffu, pid_cur, kr.head / P);
           const int slot = kr.head % P;
@@ -692,7 +697,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
         consume_tile<D, true>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+        if (w_tok == nq - 1 && lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
       }
       (void)ok;
       (void)ctx;
@@ -746,6 +751,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");  // scratch may be rewritten
+     }
     }
   }
 }
@@ -757,7 +763,7 @@ cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const Dec
   auto kern = decode_ring_kernel<D, P>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
-  const int n_items = p.b.B * p.m.Hkv * p.nq;
+  const int n_items = p.b.B * p.m.Hkv;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_items < 2 * h->num_sms ? n_items : 2 * h->num_sms, 1, 1);
   cfg.blockDim = dim3(128, 1, 1);
@@ -1039,10 +1045,11 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, cudaStream_t s) {
+cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
+                                   cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
   if (p.nq < 1 || p.nq > 4) return cudaErrorInvalidValue;
-  if (p.is_swa) return hswa_launch_decode(h, tm_pool, p, false, s);  // rings: one work item per (ring, token)
+  if (p.is_swa) return hswa_launch_decode(h, tm_pool, p, early_start, s);  // rings: one work item per (ring, token)
   const int D = p.m.D, P = p.m.P;
   if (D == 128 && P == 64) return launch_mtp_t<128, 64, 3>(tm_pool, p, s);
   if (D == 128 && P == 32) return launch_mtp_t<128, 32, 3>(tm_pool, p, s);

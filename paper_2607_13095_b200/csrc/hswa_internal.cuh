@@ -112,7 +112,7 @@ cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool,
                                cudaStream_t s);
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
 cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
-                                   cudaStream_t s);
+                                   bool early_start, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
 bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
