@@ -160,8 +160,10 @@ hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* lay
  * q: device bf16 [B][q_len][Hq][D]; k_new, v_new: device bf16 [B][q_len][Hkv][D] (required); out: device
  * [B][q_len][Hq][D]; lse: device fp32 [B][q_len][Hq] or NULL.  Token i of request r has position ctx[r] + i
  * and attends causally (to the cache and to new tokens 0..i; on SWA layers inside its own window).  The q_len
- * tokens are appended first (on a ring that is exact for q_len <= C - W + 1, checked), then one kernel streams
- * the KV once for all q_len tokens.  Workspace: as hswa_decode_attn with max_total_q = max_batch * q_len.
+ * tokens end up appended (on a ring that requires q_len <= C - W + 1, checked: HSWA_ERR_INVALID_ARG): on Full
+ * layers by an append launch ahead of one kernel that streams the KV once for all q_len tokens, on SWA layers
+ * inside the attention kernel, which stages a ring once and walks it once per token.  Workspace: as
+ * hswa_decode_attn with max_total_q = max_batch * q_len.
  * After the step call hswa_step_advance with a q_indptr describing the ACCEPTED tokens per request. */
 hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, int32_t q_len,
                                  const void* q, const void* k_new, const void* v_new, void* out, float* lse,
