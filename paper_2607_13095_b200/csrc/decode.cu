@@ -481,8 +481,12 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
 // stage buffers (metadata of the next ring fetched one ring ahead), the consumer warps prefetch the next
 // ring's Q while they work, and every ring's warps merge through a small scratch area.  The loads of ring
 // k + 1 thus overlap the compute, merge and output of ring k.
-template <int D, int P>
-__global__ void __launch_bounds__(128, 2)
+// TOKENS = false: one new token per request (nq = 1), three consumer warps take one tile each and merge.
+// TOKENS = true: a decode step that carries draft tokens (nq = 2 .. 4): one consumer warp per token walks all the
+// tiles of the ring with its own Q, mask and softmax state, so the ring is staged once for all tokens and nothing
+// has to be merged.
+template <int D, int P, bool TOKENS>
+__global__ void __launch_bounds__(TOKENS ? 160 : 128, 2)
 decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p, const int n_items) {
   constexpr int NS = 3, NW = 3;
   constexpr int HALVES = D / 64;
@@ -504,18 +508,17 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
   const ModelParams& M = p.m;
   const int n_tiles = (M.C + TK - 1) / TK;
   const bool fuse = p.k_new != nullptr;  // the new tokens are appended here; otherwise they are in the cache already
-  // With nq > 1 (a decode step that carries draft tokens) the ring's tiles are staged once and walked once per
-  // token: token w of a request sits at position ctx + w in slot ring_head + w, so it sees the ring exactly as a
-  // single new token of a request with ctx + w cached tokens and that ring head would (later drafts lie ahead of
-  // its slot, more than W - 1 slots "back" around the ring, because nq <= C - W + 1).  When the append is fused,
-  // the pass of token w patches row w into the staged tile (rows 0 .. w - 1 are there from the earlier passes)
-  // and writes it to the cache.
-  const int nq = p.nq;
+  // Token w of a request sits at position ctx + w in slot ring_head + w, so it sees the ring exactly as a single
+  // new token of a request with ctx + w cached tokens and that ring head would (later drafts lie ahead of its
+  // slot, more than W - 1 slots "back" around the ring, because nq <= C - W + 1).  When the append is fused,
+  // the warp of token w patches row w into the staged tile and writes it to the cache; a barrier among the
+  // token warps makes all nq rows visible before any of them reads the tiles.
+  const int nq = TOKENS ? p.nq : 1;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(smem_u32(&bars[i]), 1);
-      mbar_init(smem_u32(&bars[NS + i]), 1);
+      mbar_init(smem_u32(&bars[NS + i]), TOKENS ? nq : 1);  // consumers that release a tile: one per token, or its one warp
     }
     mbar_fence_init();
     tma_prefetch_desc(&tm_pool);
@@ -598,6 +601,134 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         __syncwarp();
       }
     }
+  } else if constexpr (TOKENS) {
+    // ---------------- consumers: one warp per draft token ----------------
+    const int w_tok = warp - 1;
+    if (w_tok < nq) {
+      const int g_row = lane >> 2;
+      const int qd = (lane & 3) * 2;
+      int it = blockIdx.x;
+      uint32_t qn[KS][2];
+      int ctx_n = 0, head_n = 0, pid_n = -1;
+      static_assert(2 * CHUNKS <= 32, "one chunk of the new K/V row per lane");
+      uint4 an = make_uint4(0, 0, 0, 0);
+      auto prefetch_meta = [&](int item) {  // constant during a step: may be read before the dependency wait
+        const int r = item / M.Hkv;
+        ctx_n = p.b.ctx_len[r];
+        head_n = p.b.ring_head[r];
+        pid_n = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
+      };
+      auto prefetch_qkv = [&](int item) {
+        const int r = item / M.Hkv, kh = item % M.Hkv;
+        const __nv_bfloat16* qrow = p.q + (((int64_t)r * nq + w_tok) * M.Hq + kh * M.G + g_row) * D;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          qn[ks][0] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+          qn[ks][1] = g_row < M.G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+        }
+        if (fuse && lane < 2 * CHUNKS)
+          an = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) +
+                                               (((int64_t)r * nq + w_tok) * M.Hkv + kh) * D + (lane % CHUNKS) * 8);
+      };
+      if (it < n_items) prefetch_meta(it);
+      griddep_wait();  // q, k_new, v_new and out may belong to the previous kernel on the stream
+      griddep_launch_dependents();
+      if (it < n_items) prefetch_qkv(it);
+      for (int k = 0; it < n_items; ++k, it += gridDim.x) {
+        const int r = it / M.Hkv, kh = it % M.Hkv;
+        uint32_t qf[KS][2];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          qf[ks][0] = qn[ks][0];
+          qf[ks][1] = qn[ks][1];
+        }
+        KeyRange kr;
+        kr.is_swa = 1;
+        kr.span = M.C;
+        kr.head = math_mod(head_n + w_tok, M.C);
+        kr.ctx = ctx_n + w_tok;
+        kr.W = M.W;
+        kr.C = M.C;
+        const uint4 a_cur = an;
+        const int pid_cur = pid_n;
+        if (it + gridDim.x < n_items) {
+          prefetch_meta(it + gridDim.x);
+          prefetch_qkv(it + gridDim.x);
+        }
+        // every tile of the ring is staged before this token's row is patched in and before anything is read
+        bool ok = true;
+        for (int t = 0; t < n_tiles; ++t) {
+          const int g = k * n_tiles + t;
+          if (!mbar_wait(smem_u32(&bars[g % NS]), (g / NS) & 1)) {
+            if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
+            ok = false;
+          }
+        }
+        if (fuse && ok) {
+          const int t_new = kr.head / TK, row = kr.head % TK;
+          uint8_t* sK = smem + ((k * n_tiles + t_new) % NS) * STAGE_BYTES;
+          uint8_t* sV = sK + HALVES * HALF_BYTES;
+          const int page = __shfl_sync(0xffffffffu, pid_cur, kr.head / P);
+          const bool page_ok = page >= 0 && page < p.num_pages;
+          if (!page_ok && lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, page);
+          if (lane < 2 * CHUNKS) {
+            const int kv = lane / CHUNKS, ch = lane % CHUNKS;
+            *reinterpret_cast<uint4*>((kv == 0 ? sK : sV) + (ch >> 3) * HALF_BYTES + swz128(row, ch & 7)) = a_cur;
+            if (page_ok)
+              *reinterpret_cast<uint4*>(p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * P + kr.head % P) * D + ch * 8) = a_cur;
+          }
+          fence_proxy_async_smem();
+        }
+        if (fuse) asm volatile("bar.sync 1, %0;" ::"r"(nq * 32) : "memory");  // all nq rows are in the tiles now
+        float m_run[2] = {-INFINITY, -INFINITY};
+        float l_run[2] = {0.f, 0.f};
+        float o[KS][4];
+#pragma unroll
+        for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        for (int t = 0; t < n_tiles; ++t) {
+          const int stage = (k * n_tiles + t) % NS;
+          if (ok) {
+            uint8_t* sV = smem + stage * STAGE_BYTES + HALVES * HALF_BYTES;
+            const uint32_t aK = smem_base + stage * STAGE_BYTES;
+            const uint32_t aV = aK + HALVES * HALF_BYTES;
+            const int tile_lo = t * TK;
+            const uint32_t vm0 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + lane));
+            const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
+            consume_tile<D, true>(sV, aK, aV, vm0, vm1, false, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+        }
+#pragma unroll
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+          l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+          l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+        }
+        // this warp owns the whole result of its token: straight from the accumulator fragments to the output
+        // (thread: heads qd, qd + 1; head dims 16 mt + lane / 4 and + 8)
+        if (ok) {
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (qd + j >= M.G) continue;
+            const float inv = l_run[j] > 0.f ? 1.f / l_run[j] : 0.f;
+            const int64_t row = ((int64_t)r * nq + w_tok) * M.Hq + kh * M.G + qd + j;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+              const int d0 = mt * 16 + (lane >> 2);
+              if (M.out_fp32) {
+                reinterpret_cast<float*>(p.out)[row * D + d0] = o[mt][j] * inv;
+                reinterpret_cast<float*>(p.out)[row * D + d0 + 8] = o[mt][2 + j] * inv;
+              } else {
+                reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d0] = __float2bfloat16_rn(o[mt][j] * inv);
+                reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d0 + 8] = __float2bfloat16_rn(o[mt][2 + j] * inv);
+              }
+            }
+            if ((lane >> 2) == 0 && p.lse)
+              p.lse[row] = l_run[j] > 0.f ? (m_run[j] + log2f(l_run[j])) * 0.6931471805599453f : -INFINITY;
+          }
+        }
+      }
+    }
   } else {
     // ---------------- consumers ----------------
     const int cw = warp - 1;
@@ -638,7 +769,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       const int r = it / M.Hkv, kh = it % M.Hkv;
       const int ctx0 = ctx_n, head0 = head_n, pid_cur = pid_n;
       if (it + gridDim.x < n_items) prefetch_meta(it + gridDim.x);
-     for (int w_tok = 0; w_tok < nq; ++w_tok) {
+      constexpr int w_tok = 0;  // this path serves one new token per request
       uint32_t qf[KS][2];
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -654,10 +785,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       kr.C = M.C;
       const int ctx = kr.ctx;
       const uint4 a_cur = an;
-      if (w_tok + 1 < nq)
-        prefetch_qkv(it, w_tok + 1);
-      else if (it + gridDim.x < n_items)
-        prefetch_qkv(it + gridDim.x, 0);
+      if (it + gridDim.x < n_items) prefetch_qkv(it + gridDim.x, 0);
 
       float m_run[2] = {-INFINITY, -INFINITY};
       float l_run[2] = {0.f, 0.f};
@@ -667,7 +795,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
       bool ok = true;
       for (int t = cw; t < n_tiles; t += NW) {
         const int g = k * n_tiles + t, stage = g % NS;
-        if (w_tok == 0 && !mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {  // later passes reuse the staged tile
+        if (!mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {
           if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
           ok = false;
           break;
@@ -697,7 +825,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         const uint32_t vm1 = __ballot_sync(0xffffffffu, kr.valid(tile_lo + 32 + lane));
         consume_tile<D, true>(sV, aK, aV, vm0, vm1, wrote, qf, M.scale_log2, m_run, l_run, o, lane, vm0, vm1);
         __syncwarp();
-        if (w_tok == nq - 1 && lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+        if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
       }
       (void)ok;
       (void)ctx;
@@ -751,7 +879,6 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
         if (d == 0 && p.lse) p.lse[row] = L > 0.f ? (mm + log2f(L)) * 0.6931471805599453f : -INFINITY;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory");  // scratch may be rewritten
-     }
     }
   }
 }
@@ -760,13 +887,14 @@ template <int D, int P>
 cudaError_t launch_ring_t(const hswa_handle* h, const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
   constexpr int SMEM = 3 * STAGE_BYTES + 3 * 8 * D * 4 + 3 * 8 * 2 * 4 + 1024;
-  auto kern = decode_ring_kernel<D, P>;
+  const bool tokens = p.nq > 1;
+  auto kern = tokens ? decode_ring_kernel<D, P, true> : decode_ring_kernel<D, P, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   const int n_items = p.b.B * p.m.Hkv;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_items < 2 * h->num_sms ? n_items : 2 * h->num_sms, 1, 1);
-  cfg.blockDim = dim3(128, 1, 1);
+  cfg.blockDim = dim3(tokens ? 160 : 128, 1, 1);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
