@@ -428,6 +428,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const DecodeParams p) {
   const int lane = threadIdx.x & 31;
   const ModelParams& M = p.m;
   griddep_launch_dependents();  // the next attention kernel may start its cache loads now
+  griddep_wait();               // launched early behind the kernel that writes the partials
   if (warp_global >= p.b.B * p.nq * M.Hq) return;
   const int r = warp_global / (p.nq * M.Hq);
   const int64_t row = warp_global;
@@ -1166,11 +1167,17 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s) {
   const int rows = p.b.B * p.nq * p.m.Hq;
   if (rows == 0) return cudaSuccess;
   const int blocks = (rows * 32 + 127) / 128;
-  if (p.m.D == 128)
-    combine_kernel<128><<<blocks, 128, 0, s>>>(p);
-  else
-    combine_kernel<64><<<blocks, 128, 0, s>>>(p);
-  return cudaGetLastError();
+  // programmatic dependent launch: the blocks are resident (and wait) by the time the partials are complete
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return p.m.D == 128 ? cudaLaunchKernelEx(&cfg, combine_kernel<128>, p) : cudaLaunchKernelEx(&cfg, combine_kernel<64>, p);
 }
 
 cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
