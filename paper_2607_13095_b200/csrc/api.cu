@@ -319,7 +319,8 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
     if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->batch, 16, &tq, 8)) != HSWA_OK) return st;
     if (hswa_launch_decode_prefix(tm, tq, pp, prefix_slices, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   }
-  if (hswa_launch_decode(h, tm, p, early && !cascade, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  // behind the shared-prefix stage the suffix kernel may always start early: that stage writes only its own partial slots
+  if (hswa_launch_decode(h, tm, p, early || cascade, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   if (k_new != nullptr) {
     h->chain_ok = 1;

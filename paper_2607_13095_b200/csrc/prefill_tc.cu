@@ -196,6 +196,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   int r, b, t0, n, ctx, head, h0, page_off = 0;
   TileSeq seq;
   if constexpr (PREFIX) {
+    // the suffix decode kernel that follows on the stream reads nothing this kernel writes before its own
+    // dependency wait: let it start its table reads and loads now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // blockIdx.x = slice of the prefix, blockIdx.z = group of 32 requests (16 per Q tile)
     r = blockIdx.z * 32;
     if (r >= p.b.B) return;
