@@ -177,7 +177,8 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
  * budget, or inside a section where an allocation (and the device-wide synchronisation it implies) is not
  * allowed, and that therefore has no workspace to offer.
  *   - Limit: a batch whose partials need more than HSWA_STATIC_WS_BYTES (roughly B * Hq * ceil((max_ctx_len
- *     + 1) / 2048) * (4 * D + 8) bytes on a Full layer; SWA layers need none) is rejected with
+ *     + 1) / 4096) * (4 * D + 8) bytes on a Full layer, more for small batches, which get shorter splits;
+ *     SWA layers need none) is rejected with
  *     HSWA_ERR_WORKSPACE and nothing is launched.
  *   - Every GPU that loads the library holds the array until the process exits.
  *   - The first call on a device looks up the array's device address (with that device current, which must be
