@@ -4,9 +4,12 @@
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg4|cfg5|cfg3] [--impl reference]
 
 A "step" is one pass of the whole hot path over one synthetic batch: for every layer of the stack the fused
-KV append + attention (+ split combine), then the step advance.  The default workload is the decode block of
-6 SWA + 1 Full layers, batch 64, contexts U[4k, 32k] (the configuration the headline metric is quoted on);
-the default run also reports, under "extra", the chunked-prefill block (8 x 8192-token chunks).
+KV append + attention (+ split combine), then the step advance.  The default workload is the largest
+single-GPU configuration: the full-stack long-context decode step (70 layers = 60 SWA + 10 Full, batch 16,
+contexts U[64k, 256k], 100 GB of KV per step).  The default run also reports, under "extra", the other named
+configurations, each with its own warm-up, >= 20 timed steps and clock record: the 7-layer decode block at batch 64
+(one token per request, and 4 tokens per request through the multi-token entry point), the prefix-hit decode
+(plain and cascade, against logical and unique bytes) and the chunked-prefill block (per-layer-kind rooflines).
 One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs its own batch (weak scaling, no
 data-path collective) and the time is the max over ranks.
 """
@@ -34,13 +37,13 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep", "prefetch", "buckets"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg2", "cfg3", "cfg4", "cfg5", "prefix_sweep", "prefetch", "buckets"])
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (cfg5: fewer to fit)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (smaller cases for profiling)")
     ap.add_argument("--chunk", type=int, default=0, help="cfg3: override the prefill chunk length")
     ap.add_argument("--mtp", type=int, default=1, help="decode q_len per request (2-4: hswa_decode_attn_mtp)")
     ap.add_argument("--cascade", action="store_true", help="cfg4: use hswa_decode_attn_shared_prefix on the shared prefix")
-    ap.add_argument("--no-extra", action="store_true", help="skip the prefill block reported under 'extra'")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations reported under 'extra'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="run the end-to-end step eagerly instead of as a CUDA graph")
@@ -165,7 +168,8 @@ class DecodeBench:
         self.ctx0, self.head0 = i32(t.ctx_len), i32(t.ring_head)
         self.ctx, self.head = self.ctx0.clone(), self.head0.clone()
         B = t.batch
-        self.max_ctx = int(t.ctx_len.max()) + total_steps + 1 + mtp
+        # bound of ctx_len over the run: one accepted token per step; the tables above cover max_ctx + mtp positions
+        self.max_ctx = int(t.ctx_len.max()) + total_steps
         self.batch = hb.Batch(self.ctx, i32(t.block_table), i32(t.ring_table), self.head, None, max_q_len=1,
                               total_q=B, max_ctx_len=self.max_ctx)
         ws_bytes = hb.hswa_workspace_bytes(self.h, B, B * mtp, self.max_ctx)
@@ -252,59 +256,146 @@ def time_events(torch, fn, warmup, steps):
     return e0.elapsed_time(e1) / steps
 
 
-def prefill_extra(device, peaks):
-    """Chunked-prefill block (8 requests x 8192 new tokens over cached contexts U[0, 16k]): per-layer-kind time."""
+def stats(xs):
+    xs = np.asarray(xs, dtype=np.float64)
+    return {"mean": float(xs.mean()), "median": float(np.median(xs)), "min": float(xs.min()), "max": float(xs.max()),
+            "n": int(xs.size)}
+
+
+def time_launches(torch, fn, warmup, n, index):
+    """n separately timed calls of fn (CUDA events on the current stream) after `warmup` untimed ones, with the SM
+    clock sampled meanwhile.  Returns (per-call ms list, clock summary)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    with ClockSampler(index) as clocks:
+        for a, b in ev:
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev], clocks.summary()
+
+
+def prefill_extra(device, peaks, index=0, launches=20):
+    """Chunked-prefill block (8 requests x 8192 new tokens over cached contexts U[0, 16k]): each layer kind timed
+    over `launches` separately timed layer calls (attention + append) after 3 warm-ups, with its own roofline
+    object and clock record.  Inputs (Q 1.07 GB, chunk K/V 0.27 GB, output 1.07 GB) are larger than L2."""
     import torch
     from paper_2607_13095_b200 import accounting
+    from paper_2607_13095_b200 import binding as hb
     w = make_workload("cfg3")
     pb = PrefillBench(w, device)
     full_i = w.layer_is_swa.index(False)
     swa_i = w.layer_is_swa.index(True)
-    ms_full = time_events(torch, lambda: pb.run_layer(full_i), 2, 5)
-    ms_swa = time_events(torch, lambda: pb.run_layer(swa_i), 2, 5)
+    ms_full, clk_full = time_launches(torch, lambda: pb.run_layer(full_i), 3, launches, index)
+    ms_swa, clk_swa = time_launches(torch, lambda: pb.run_layer(swa_i), 3, launches, index)
+    # the SWA layer again right behind a Full layer, i.e. at the clock the Full layer leaves behind (as in the block)
+    ms_swa_in_block = []
+    for _ in range(5):
+        pb.run_layer(full_i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        pb.run_layer(swa_i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_swa_in_block.append(e0.elapsed_time(e1))
+    st = hb.hswa_get_async_error(pb.h)
+    if st[0] != hb.HSWA_OK:
+        raise SystemExit(f"device error word set during the prefill block: {st}")
+    sf, ss = stats(ms_full), stats(ms_swa)
     f_full, f_swa = accounting.prefill_flops(w, False), accounting.prefill_flops(w, True)
+    b_swa = accounting.prefill_compulsory_bytes(w, True)
     n_full = sum(1 for s in w.layer_is_swa if not s)
     n_swa = len(w.layer_is_swa) - n_full
-    block_ms = n_full * ms_full + n_swa * ms_swa
-    tf_full = f_full / (ms_full * 1e-3) / 1e12
+    swa_blk = float(np.median(ms_swa_in_block))
+    block_ms = n_full * sf["mean"] + n_swa * swa_blk
+    tf = f_full / (sf["mean"] * 1e-3) / 1e12
+    gbs = b_swa / (ss["mean"] * 1e-3) / 1e9
     return {
-        "workload": w.name, "full_layer_ms": ms_full, "swa_layer_ms": ms_swa,
-        "full_layer_tflops": tf_full, "swa_layer_tflops": f_swa / (ms_swa * 1e-3) / 1e12,
-        "block_tflops": (n_full * f_full + n_swa * f_swa) / (block_ms * 1e-3) / 1e12,
+        "workload": w.name, "launches_timed": launches, "warmup": 3,
+        "full_layer_ms": sf["mean"], "full_layer_ms_stats": sf, "swa_layer_ms": ss["mean"], "swa_layer_ms_stats": ss,
+        "swa_layer_ms_behind_full_layer": swa_blk,
+        "full_layer_tflops": tf, "swa_layer_tflops": f_swa / (ss["mean"] * 1e-3) / 1e12,
+        "block_ms": block_ms, "block_tflops": (n_full * f_full + n_swa * f_swa) / (block_ms * 1e-3) / 1e12,
         "block_tokens_per_s": w.tables.total_q / (block_ms * 1e-3),
-        "full_layer_frac_of_measured_bf16_peak": tf_full / peaks["bf16_tflops"],
-        "full_layer_frac_of_nominal_bf16_peak": tf_full / 2250.0,
+        "full_layer_roofline": {
+            "bound": "tensor", "achieved": tf, "unit": "TFLOP/s", "peak": peaks["bf16_tflops"],
+            "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (cuBLAS bf16 burst)",
+            "frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
+            "ms_per_launch": sf["mean"], "algorithmic_flops_per_launch": f_full,
+            "traffic": stored_traffic("prefill_full_cfg3"),
+            "kernel": "prefill_tc_kernel + append_kernel, one Full layer", "clocks": clk_full},
+        "swa_layer_roofline": {
+            "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "frac_of_nominal_8TBs": gbs / 8000.0, "ms_per_launch": ss["mean"],
+            "algorithmic_bytes_per_launch": b_swa, "traffic": stored_traffic("prefill_swa_cfg3"),
+            "kernel": "SWA prefill kernels + append_ring_kernel, one SWA layer", "clocks": clk_swa},
     }
 
 
 # ---------------------------------------------------------------------------------------------------------
-def oracle_decode_sample(w, layers_pools_host, q_host, k_host, v_host, t, n_full_rows, seed=0):
-    """Time the CPU oracle on a bounded sample of the decode workload and extrapolate to a whole step.
-    Returns (estimated seconds per step, description, threads)."""
+def pick_requests(t, n):
+    """A bounded sample of requests: the longest, the shortest and evenly spaced others (deterministic)."""
+    order = np.argsort(t.ctx_len, kind="stable")
+    idx = {int(order[-1]), int(order[0])}
+    for k in np.linspace(0, t.batch - 1, num=max(n, 2)):
+        if len(idx) >= n:
+            break
+        idx.add(int(order[int(round(k))]))
+    return np.array(sorted(idx), dtype=np.int64)
+
+
+def compact_tables(t, d, reqs):
+    """Block and ring tables of the requests `reqs` renumbered onto compact pools that hold only their pages.
+    Returns (block_table, full page ids in compact order, ring_table, ring page ids in compact order).  Pure
+    bookkeeping: which physical page sits where; pages shared between requests are kept once."""
+    need = [-(-(int(t.ctx_len[r]) + 1) // d.page_size) for r in reqs]
+    full_ids, remap = [], {}
+    bt = np.zeros((len(reqs), max(need)), dtype=np.int32)
+    for i, r in enumerate(reqs):
+        for j in range(need[i]):
+            pg = int(t.block_table[r, j])
+            if pg not in remap:
+                remap[pg] = len(full_ids)
+                full_ids.append(pg)
+            bt[i, j] = remap[pg]
+    ring_ids = t.ring_table[reqs].reshape(-1)
+    rt = np.arange(ring_ids.size, dtype=np.int32).reshape(len(reqs), -1)
+    return bt, np.array(full_ids, dtype=np.int64), rt, ring_ids.astype(np.int64)
+
+
+def oracle_decode_sample(w, t, reqs, bt, full_pool, rt, ring_pool, q, k, v, heads_full=None):
+    """Time the CPU oracle, as it stands, on all (or `heads_full`) query heads of the requests `reqs` for one Full
+    and one SWA layer, and extrapolate to a whole step by key count.  Pools and tables are the compact ones of
+    compact_tables; q, k, v hold only those requests.  Returns (estimated seconds per step, description, threads,
+    measured seconds)."""
     from oracle import hswa_oracle as orc
     d = w.dims
     cfg = orc.OracleConfig(d.num_q_heads, d.num_kv_heads, d.head_dim, d.page_size, d.window, d.ring_pages)
-    ob = orc.OracleBatch(t.ctx_len, t.block_table, t.ring_table, t.ring_head)
-    rng = np.random.default_rng(seed)
-    est = 0.0
-    desc = []
-    for is_swa, pool, count in layers_pools_host:
-        B, Hq = t.batch, d.num_q_heads
-        all_rows = B * Hq
-        n = min(all_rows, n_full_rows if not is_swa else all_rows)
-        pick = rng.choice(all_rows, size=n, replace=False)
-        tok, head = (pick // Hq).astype(np.int32), (pick % Hq).astype(np.int32)
-        keys = np.minimum(t.ctx_len + 1, d.window) if is_swa else t.ctx_len + 1
+    ob = orc.OracleBatch(t.ctx_len[reqs], bt, rt, t.ring_head[reqs])
+    n_full = sum(1 for s in w.layer_is_swa if not s)
+    n_swa = len(w.layer_is_swa) - n_full
+    est, spent, desc = 0.0, 0.0, []
+    for is_swa, pool, count in ((False, full_pool, n_full), (True, ring_pool, n_swa)):
+        Hq = d.num_q_heads
+        heads = np.arange(Hq) if (is_swa or heads_full is None) else np.asarray(heads_full)
+        tok = np.repeat(np.arange(len(reqs)), len(heads)).astype(np.int32)
+        head = np.tile(heads, len(reqs)).astype(np.int32)
+        keys = np.minimum(t.ctx_len.astype(np.int64) + 1, d.window) if is_swa else t.ctx_len.astype(np.int64) + 1
         total_keys = float(keys.sum()) * Hq
-        sample_keys = float(keys[tok].sum())
+        sample_keys = float(keys[reqs].sum()) * len(heads)
         layer = orc.OracleLayer(pool, is_swa)
         t0 = time.perf_counter()
-        orc.attention(cfg, layer, ob, q_host, k_host, v_host, rows=(tok, head))
+        orc.attention(cfg, layer, ob, q, k, v, rows=(tok, head))
         dt = time.perf_counter() - t0
+        spent += dt
         est += dt * (total_keys / max(sample_keys, 1.0)) * count
-        desc.append(f"{'swa' if is_swa else 'full'} layer: {n} of {all_rows} (request, head) rows in {dt:.2f}s, "
-                    f"scaled by keys x{total_keys / max(sample_keys, 1.0):.2f} and x{count} layers")
-    return est, "; ".join(desc), orc.num_threads()
+        desc.append(f"{'swa' if is_swa else 'full'} layer: {len(tok)} of {t.batch * Hq} (request, head) rows "
+                    f"({len(reqs)} requests x {len(heads)} heads) in {dt:.2f}s, scaled by keys "
+                    f"x{total_keys / max(sample_keys, 1.0):.2f} and x{count} layers")
+    return est, "; ".join(desc), orc.num_threads(), spent
 
 
 def host_bits(t):
@@ -312,59 +403,82 @@ def host_bits(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def cpu_baseline_decode(bench, rows=2048):
-    w, t = bench.w, bench.t
-    n_full = sum(1 for s in w.layer_is_swa if not s)
-    n_swa = len(w.layer_is_swa) - n_full
-    fi = bench.full_idx[0]
-    si = w.layer_is_swa.index(True)
-    pools = [(False, host_bits(bench.layers[fi].pool), n_full), (True, host_bits(bench.layers[si].pool), n_swa)]
-    est, desc, threads = oracle_decode_sample(w, pools, host_bits(bench.q[fi]), host_bits(bench.k_new[fi]),
-                                              host_bits(bench.v_new[fi]), t, rows)
-    return {"value": t.batch / est, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+def cpu_baseline_decode(bench, n_requests=4):
+    """The oracle on a bounded sample of the bench's own device state (the pages of a few requests are gathered on
+    the device and copied to the host, so a 10 GB pool never crosses PCIe whole)."""
+    import torch
+    w, t, d = bench.w, bench.t, bench.w.dims
+    fi, si = bench.full_idx[0], w.layer_is_swa.index(True)
+    reqs = pick_requests(t, min(n_requests, t.batch))
+    bt, full_ids, rt, ring_ids = compact_tables(t, d, reqs)
+    dev = bench.layers[fi].pool.device
+    full_pool = host_bits(bench.layers[fi].pool.index_select(0, torch.from_numpy(full_ids).to(dev)))
+    ring_pool = host_bits(bench.layers[si].pool.index_select(0, torch.from_numpy(ring_ids).to(dev)))
+    ridx = torch.from_numpy(reqs).to(dev)
+    q, k, v = (host_bits(x[fi].index_select(0, ridx)) for x in (bench.q, bench.k_new, bench.v_new))
+    est, desc, threads, spent = oracle_decode_sample(w, t, reqs, bt, full_pool, rt, ring_pool, q, k, v)
+    return {"value": t.batch / est, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+            "extrapolated": True, "measured_seconds": spent}
 
 
 # ---------------------------------------------------------------------------------------------------------
 def run_reference(args):
-    """The reference arm: the fp64 CPU oracle, as it stands, on the host cores, on a bounded sample per step."""
+    """The reference arm: the fp64 CPU oracle, as it stands, on the host cores.  Each step times a bounded sample
+    of the workload (a few requests, a few heads of the Full layer, every head of an SWA layer) and extrapolates to
+    the whole step by key count; the line says so ("extrapolated") and gives the seconds actually measured."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import torch
     from paper_2607_13095_b200 import workloads as wl
     w = make_workload(args.workload if args.workload != "cfg3" else "cfg2", layers=args.layers, batch=args.batch)
     d, t = w.dims, w.tables
-    # host-only state: one Full and one SWA pool; a random 64-page block repeated (the values do not affect time)
+    reqs = pick_requests(t, min(3, t.batch))
+    bt, full_ids, rt, ring_ids = compact_tables(t, d, reqs)
+
+    # host-only state: compact pools filled by repeating a random 64-page block (the values do not affect time)
     def rand_pool(n_pages, seed):
         base = wl.bf16_bits_normal(seed, (min(n_pages, 64), 2, d.num_kv_heads, d.page_size, d.head_dim))
         return np.resize(base, (n_pages,) + base.shape[1:])
-    n_full = sum(1 for s in w.layer_is_swa if not s)
-    n_swa = len(w.layer_is_swa) - n_full
-    # the Full pool only needs the pages the sampled requests touch; keep it whole when it is small
-    pools = [(False, rand_pool(t.num_full_pages, 11), n_full), (True, rand_pool(t.num_ring_pages, 12), n_swa)]
-    q = wl.bf16_bits_normal(13, (t.batch, d.num_q_heads, d.head_dim))
-    k = wl.bf16_bits_normal(14, (t.batch, d.num_kv_heads, d.head_dim))
-    v = wl.bf16_bits_normal(15, (t.batch, d.num_kv_heads, d.head_dim))
-    rows = 256
-    ests = []
+    full_pool, ring_pool = rand_pool(len(full_ids), 11), rand_pool(len(ring_ids), 12)
+    q = wl.bf16_bits_normal(13, (len(reqs), d.num_q_heads, d.head_dim))
+    k = wl.bf16_bits_normal(14, (len(reqs), d.num_kv_heads, d.head_dim))
+    v = wl.bf16_bits_normal(15, (len(reqs), d.num_kv_heads, d.head_dim))
+    # heads of the Full layer per step: about 5e7 (row, key) pairs, i.e. a second or two on a few cores
+    keys = float((t.ctx_len[reqs].astype(np.int64) + 1).sum())
+    n_heads = int(min(d.num_q_heads, max(1, round(5e7 / keys))))
+    ests, spents = [], []
     desc, threads = "", 1
     for i in range(args.warmup + args.steps):
-        est, desc, threads = oracle_decode_sample(w, pools, q, k, v, t, rows, seed=i)
+        heads = (np.arange(n_heads) * (d.num_q_heads // n_heads) + i) % d.num_q_heads
+        est, desc, threads, spent = oracle_decode_sample(w, t, reqs, bt, full_pool, rt, ring_pool, q, k, v, heads_full=heads)
         if i >= args.warmup:
             ests.append(est)
+            spents.append(spent)
     sec = float(np.mean(ests))
     val = t.batch / sec
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "layers": len(w.layer_is_swa), "batch": t.batch,
-                   "note": "CPU oracle timed on a bounded sample per step and extrapolated by key count"},
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "extrapolated": True,
+        "measured_seconds_per_step_sample": float(np.mean(spents)),
+        "config": workload_config(w, t, False, 1) | {
+            "note": "CPU oracle timed on a bounded sample per step and extrapolated by key count; ms_per_step is that "
+                    "estimate, measured_seconds_per_step_sample the time each step's sample really took"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def workload_config(w, t, cascade, mtp):
+    d = w.dims
+    return {"workload": w.name, "layers": len(w.layer_is_swa), "swa_layers": int(sum(w.layer_is_swa)),
+            "batch": t.batch, "num_q_heads": d.num_q_heads, "num_kv_heads": d.num_kv_heads,
+            "head_dim": d.head_dim, "page_size": d.page_size, "window": d.window,
+            "ctx_sum": int(t.ctx_len.astype(np.int64).sum()), "shared_prefix_tokens": t.shared_prefix_pages * d.page_size,
+            "cascade": bool(cascade), "mtp_q_len": mtp, "l2": "inputs larger than L2 (Full-layer KV streamed per step "
+            "exceeds 126 MB and evicts the SWA rings between reuses)", "out_dtype": "bf16"}
 
 
 def run_prefix_sweep(args, torch, device, peaks):
@@ -573,6 +687,118 @@ def run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks):
     print(json.dumps(line))
 
 
+def read_stream_gbs(torch, device):
+    """A plain read-only stream over 4 GiB (torch.sum), best of 5: what this machine's HBM gives a kernel that only reads,
+    which is what decode attention does; reported beside the copy-based measured peak."""
+    x = torch.empty(2 << 30, dtype=torch.bfloat16, device=device)
+    x.zero_()
+    best = float("inf")
+    for _ in range(7):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        x.sum()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    return x.numel() * 2 / (best * 1e-3) / 1e9
+
+
+def measure_decode(bench, steps, warmup, index, barrier, world=1, dist=None):
+    """Warm-up, then EXACTLY `steps` steps between two events (with barrier + synchronize on both sides); the first
+    Full layer of every step is bracketed by its own events (the dominant kernel's launch time), every step by its
+    own pair too (spread).  Returns a dict of times in ms and the clock record."""
+    import torch
+    from paper_2607_13095_b200 import binding as hb
+    for _ in range(warmup):
+        bench.step()
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    with ClockSampler(index) as clocks:
+        marks[0].record()
+        for k in range(steps):
+            bench.step(ev[k])
+            marks[k + 1].record()
+        torch.cuda.synchronize()
+    barrier()
+    st = hb.hswa_get_async_error(bench.h)
+    if st[0] != hb.HSWA_OK:
+        raise SystemExit(f"device error word set during the timed region: {st}")
+    ms_total = marks[0].elapsed_time(marks[-1])
+    tmax = torch.tensor([ms_total], device=bench.ctx.device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    per_step = [marks[k].elapsed_time(marks[k + 1]) for k in range(steps)]
+    full = [a.elapsed_time(b) for a, b in ev]
+    n_full = len(bench.full_idx)
+    n_swa = len(bench.layers) - n_full
+    ms_step = float(tmax.item()) / steps
+    return {"ms_per_step": ms_step, "ms_per_step_stats": stats(per_step), "full_layer_ms": float(np.mean(full)),
+            "full_layer_ms_stats": stats(full),
+            # what is left of a step after its Full layers, per SWA layer (includes the step advance)
+            "swa_layer_ms_derived": max(ms_step - n_full * float(np.mean(full)), 0.0) / max(n_swa, 1),
+            "clocks": clocks.summary()}
+
+
+def decode_rooflines(w, bench, m, peaks, steps, warmup, read_gbs, traffic_key=None):
+    """Roofline objects of a decode measurement: the Full-layer call against logical and unique bytes, the step."""
+    from paper_2607_13095_b200 import accounting
+    d, t = w.dims, bench.t
+    grown = t.batch * (warmup + steps // 2) * d.kv_bytes_per_token  # context growth of the run so far (mean)
+    logical = accounting.decode_layer_bytes(w, False) + grown
+    unique = accounting.decode_layer_bytes(w, False, unique=True) + grown
+    ms = m["full_layer_ms"]
+    ach_l, ach_u = logical / (ms * 1e-3) / 1e9, unique / (ms * 1e-3) / 1e9
+    shared = t.shared_prefix_pages > 0
+    # a roofline is bytes that must cross the HBM interface: with a shared prefix that is the unique figure; the
+    # logical figure (what a sharing-oblivious kernel asks for, partly served by L2) is reported beside it
+    ach = ach_u if shared else ach_l
+    roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+            "traffic": None, "kernel": "decode_kernel + combine_kernel, one Full layer"
+            + (" (+ prefill_tc_kernel<prefix> with --cascade)" if bench.shared_prefix else ""),
+            "ms_per_launch": ms, "algorithmic_bytes_per_launch": unique if shared else logical,
+            "peak_source": peaks["source"] + " (copy: read + write bytes)", "frac_of_nominal_8TBs": ach / 8000.0,
+            "frac_of_read_stream": (ach / read_gbs) if read_gbs else None, "read_stream_gbs": read_gbs}
+    if shared:
+        roof["bytes"] = "unique (the shared prefix counted once)"
+        roof["frac_unique"] = ach_u / peaks["hbm_gbs"]
+        roof["logical_gbs"] = ach_l
+        roof["frac_logical"] = ach_l / peaks["hbm_gbs"]
+        roof["logical_bytes_per_launch"] = logical
+    per_key = stored_traffic("decode_full_dram_bytes_per_kv_byte")
+    if per_key and not shared:
+        roof["traffic"] = int(per_key * logical)
+        roof["traffic_note"] = "ncu DRAM bytes of a small capture scaled by KV bytes (traffic is proportional to them)"
+    step_l = accounting.decode_algorithmic_bytes(w)
+    step_u = accounting.decode_unique_bytes(w)
+    out = {"roofline": roof, "step_gbs": step_l / (m["ms_per_step"] * 1e-3) / 1e9,
+           "step_frac_of_measured_hbm": (step_u if shared else step_l) / (m["ms_per_step"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    if shared:
+        out["step_unique_gbs"] = step_u / (m["ms_per_step"] * 1e-3) / 1e9
+        out["step_frac_logical"] = step_l / (m["ms_per_step"] * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    return out
+
+
+def decode_extra(name, device, peaks, read_gbs, index, steps=30, warmup=5, cascade=False, mtp=1, batch=0):
+    """One more decode configuration measured like the headline one (own warm-up, own clocks), as a summary dict."""
+    import torch
+    w = make_workload(name, batch=batch)
+    bench = DecodeBench(w, 2 * (steps + warmup) + 8, device, cascade=cascade, mtp=mtp)
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    m = measure_decode(bench, steps, warmup, index, barrier)
+    r = decode_rooflines(w, bench, m, peaks, steps, warmup, read_gbs)
+    tokens = bench.t.batch * mtp
+    res = {"workload": w.name, "cascade": bool(cascade), "mtp_q_len": mtp, "steps": steps, "warmup": warmup,
+           "tokens_per_s": tokens / (m["ms_per_step"] * 1e-3), **m, **r,
+           "gpu_launches": bench.launches_per_step * steps}
+    del bench
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -580,7 +806,6 @@ def main():
         return
     import torch
     import torch.distributed as dist
-    from paper_2607_13095_b200 import accounting
     from paper_2607_13095_b200 import binding as hb
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -607,6 +832,8 @@ def main():
     if args.workload == "cfg3":
         run_prefill_main(args, torch, dist, world, rank, local_rank, device, peaks)
         return
+    read_gbs = read_stream_gbs(torch, device) if world == 1 else None
+    torch.cuda.empty_cache()
     w = make_workload(args.workload, seed_offset=rank, layers=args.layers, batch=args.batch)
     total_steps = args.steps + args.warmup
     bench = DecodeBench(w, 2 * total_steps + 8, device, cascade=args.cascade, mtp=args.mtp)
@@ -619,29 +846,11 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing ----
-    for _ in range(args.warmup):
-        bench.step()
-    barrier()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local_rank) as clocks:
-        e0.record()
-        for k in range(args.steps):
-            bench.step(ev[k])
-        e1.record()
-        torch.cuda.synchronize()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    full_ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
-    st = hb.hswa_get_async_error(bench.h)
-    if st[0] != hb.HSWA_OK:
-        raise SystemExit(f"device error word set during the timed region: {st}")
-    tmax = torch.tensor([ms_total], device=device, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms_step = float(tmax.item()) / args.steps
+    m = measure_decode(bench, args.steps, args.warmup, local_rank, barrier, world, dist)
+    ms_step = m["ms_per_step"]
     tokens_per_step = t.batch * world * args.mtp  # with --mtp: query tokens scored per step (1 accepted + drafts)
     value = tokens_per_step / (ms_step * 1e-3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     # ---- end to end: pinned host inputs -> device, step, result -> host, every step ----
     e2e = None
@@ -728,31 +937,20 @@ def main():
         return
 
     # ---- roofline of the dominant kernel: Full-layer decode (split-K partial kernel + combine) ----
-    keys_full = int((t.ctx_len.astype(np.int64) + 1).sum()) + t.batch * (args.warmup + args.steps // 2)
-    per_req_io = 2 * d.num_q_heads * d.head_dim * 2 + d.kv_bytes_per_token
-    full_bytes = keys_full * d.kv_bytes_per_token + t.batch * per_req_io
-    achieved = full_bytes / (full_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": stored_traffic(f"decode_full_{args.workload}"),
-                "kernel": "decode_kernel + combine_kernel, one Full layer", "ms_per_launch": full_ms,
-                "algorithmic_bytes_per_launch": full_bytes, "peak_source": peaks["source"],
-                "frac_of_nominal_8TBs": achieved / 8000.0}
-    step_bytes = accounting.decode_algorithmic_bytes(w)
+    r = decode_rooflines(w, bench, m, peaks, args.steps, args.warmup, read_gbs)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
-        "config": {"workload": w.name, "layers": len(w.layer_is_swa), "swa_layers": int(sum(w.layer_is_swa)),
-                   "batch": t.batch, "num_q_heads": d.num_q_heads, "num_kv_heads": d.num_kv_heads,
-                   "head_dim": d.head_dim, "page_size": d.page_size, "window": d.window,
-                   "ctx_sum": int(t.ctx_len.sum()), "shared_prefix_tokens": t.shared_prefix_pages * d.page_size,
-                   "cascade": bool(args.cascade), "mtp_q_len": args.mtp, "l2": "inputs larger than L2 (Full-layer KV streamed per step "
-                   "exceeds 126 MB and evicts the SWA rings between reuses)", "out_dtype": "bf16"},
-        "step_gbs": step_bytes / (ms_step * 1e-3) / 1e9 * world,
-        "step_frac_of_measured_hbm": step_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-        "roofline": roofline, "clocks": clocks.summary(), "e2e": e2e,
+        "ms_per_step": ms_step, "ms_per_step_stats": m["ms_per_step_stats"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(w, t, args.cascade, args.mtp),
+        "full_layer_ms": m["full_layer_ms"], "swa_layer_ms_derived": m["swa_layer_ms_derived"],
+        "step_gbs": r["step_gbs"] * world, "step_frac_of_measured_hbm": r["step_frac_of_measured_hbm"],
+        "roofline": r["roofline"], "clocks": m["clocks"], "e2e": e2e,
         "gpu_launches": bench.launches_per_step * args.steps,
     }
+    for key in ("step_unique_gbs", "step_frac_logical"):
+        if key in r:
+            line[key] = r[key]
     if not args.no_graph and world == 1:
         # The same device-resident step replayed as one CUDA graph (reported separately: the host's launch time
         # matters at small batch, where a layer's kernels are shorter than the calls that launch them).
@@ -771,10 +969,17 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         bench.reset()
         line["cpu_baseline"] = cpu_baseline_decode(bench)
-    if not args.no_extra and world == 1 and args.workload == "cfg2":
+    if not args.no_extra and world == 1 and args.workload == "cfg5" and not args.layers and not args.batch:
+        # the other named configurations, one after the other on the freed device
         del bench
         torch.cuda.empty_cache()
-        line["extra"] = {"prefill": prefill_extra(device, peaks)}
+        extra = {}
+        extra["cfg2"] = decode_extra("cfg2", device, peaks, read_gbs, local_rank, steps=50)
+        extra["mtp4"] = decode_extra("cfg2", device, peaks, read_gbs, local_rank, steps=30, mtp=4)
+        extra["cfg4"] = {"plain": decode_extra("cfg4", device, peaks, read_gbs, local_rank, steps=30),
+                         "cascade": decode_extra("cfg4", device, peaks, read_gbs, local_rank, steps=30, cascade=True)}
+        extra["prefill"] = prefill_extra(device, peaks, local_rank)
+        line["extra"] = extra
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

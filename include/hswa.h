@@ -21,8 +21,11 @@
  *   - Within a step the library may overlap consecutive fused decode calls issued through one handle on one
  *     stream (programmatic dependent launch): a later kernel reads the batch arrays and its layer's pool while
  *     the earlier one drains, and waits before touching q, k_new, v_new or its outputs.  This relies on the
- *     contract below that the batch arrays are constant during a step and that only this library writes the
- *     pools; any other call on the handle (append, prefill, advance, error read) ends the overlap.
+ *     contract below that the batch arrays are constant during a step and that only this library, through this
+ *     handle, writes the pools; any other call on the handle (append, prefill, advance, error read) ends the
+ *     overlap, and two consecutive calls on the same pool never overlap.  A caller that writes a pool itself
+ *     between two decode calls of a step, or shares pools between handles, switches the overlap off with
+ *     hswa_set_overlap(h, 0).
  *   - No global mutable state except the static scratch of hswa_decode_attn_static_ws; a handle may be used
  *     from one thread at a time.
  *
@@ -109,31 +112,55 @@ typedef struct {
 hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out);
 void hswa_destroy(hswa_handle* h);
 
-/* Bytes of workspace (device memory, 256-byte aligned, caller-owned) that hswa_decode_attn and
- * hswa_prefill_attn need for batches bounded by the three arguments.  Pure host arithmetic. */
+/* Switches the overlap of consecutive fused decode calls (see Conventions) on (default) or off for this handle.
+ * Off, every kernel waits for all earlier work on the stream before it reads anything.  (No paper counterpart:
+ * a scheduling knob of this library.) */
+hswa_status hswa_set_overlap(hswa_handle* h, int32_t enabled);
+
+/* Bytes of workspace (device memory, 256-byte aligned, caller-owned) that is enough for every decode call
+ * (hswa_decode_attn, _shared_prefix, _mtp with max_total_q = max_batch * q_len) on batches bounded by the three
+ * arguments; hswa_prefill_attn needs none.  An upper bound over all smaller batches and contexts.  Pure host
+ * arithmetic. */
 size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max_total_q, int32_t max_ctx_len);
 
-/* Debug aid: checks on the device, for the given layer kind, that every id and length the step would use
- * is in range (0 <= ctx, n >= 0, block-table coverage of ctx + n, page ids < num_pages, ring_head in
- * [0, C)).  The first violation is recorded in the error word as {HSWA_ERR_BOUNDS, request, index, value}. */
+/* Exact bytes of workspace ONE decode call needs (split-K partials of paper Sec. 2.2's memory-bound decode: the
+ * key range of a Full layer is cut into splits whose (m, l, o) partials live in the workspace): the call on a
+ * layer of the given kind with batch->batch = batch, batch->max_ctx_len = max_ctx_len, the given
+ * shared_prefix_len (0 for hswa_decode_attn) and q_len (1, or 2-4 for hswa_decode_attn_mtp).  A call is accepted
+ * iff its workspace_bytes is at least this.  0 for SWA layers, for calls that need no split, and for arguments
+ * out of range.  Pure host arithmetic. */
+size_t hswa_decode_workspace_need(const hswa_handle* h, int32_t is_swa, int32_t batch, int32_t max_ctx_len,
+                                  int32_t shared_prefix_len, int32_t q_len);
+
+/* Debug aid (paper Sec. 3.1.3: attention must never read invalid or overwritten slots): checks on the device,
+ * for the given layer kind, that every id and length the step would use is in range (0 <= ctx <= max_ctx_len,
+ * 0 <= n <= max_q_len, block-table coverage of ctx + n, page ids < num_pages, ring_head in [0, C)).  The first
+ * violation is recorded in the error word as {HSWA_ERR_BOUNDS, request, index, value}; index -1 / -2 / -3 / -4
+ * name ctx, n, block-table coverage and ring head. */
 hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, void* stream);
 
 /* KV append (Sec. 3.1.1 pools; Sec. 3.1.3: an SWA pool stays at window magnitude).
  * k_new, v_new: device, bf16 [T][Hkv][D].  Token i of request r is written at the storage location of
  * position ctx[r] + i.  On an SWA layer later tokens overwrite earlier ones, so only the last min(n, C)
  * tokens of a request are written.  Nothing else in the pool changes.
- * Caller guarantees that pages receiving an append are not shared with another request. */
+ * Caller guarantees that pages receiving an append are not shared with another request.
+ * A position the block table does not cover, or a page id outside the pool, is recorded in the error word
+ * (HSWA_ERR_BOUNDS) and that row is not written. */
 hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* k_new,
                            const void* v_new, void* stream);
 
-/* Batched GQA decode attention, one new token per request (batch->q_indptr must be NULL).
+/* Batched GQA decode attention, one new token per request (batch->q_indptr must be NULL).  Paper Sec. 2.2:
+ * decode is memory-bound and its cost is the KV bytes read -- every cached token on a Full layer, the last W
+ * on an SWA layer (Sec. 2.1), found through the block table / ring of Sec. 3.1.1.
  * q: device bf16 [B][Hq][D].  out: device [B][Hq][D] in cfg.out_dtype.  lse: device fp32 [B][Hq] or NULL.
  * k_new, v_new: device bf16 [B][Hkv][D], or both NULL.
  *   non-NULL: the new token's K/V are appended (fused into the attention kernel) and attended to.
  *   NULL:     the caller already ran hswa_kv_append with the same un-advanced batch; position ctx[r] is
  *             read from the cache.
  * Full layers split the key range over thread blocks (split-K) and merge the partial results; partials
- * live in `workspace`. */
+ * live in `workspace` (hswa_decode_workspace_need bytes; too few: HSWA_ERR_WORKSPACE, nothing launched).
+ * On a Full layer the block table must cover position max_ctx_len (max_blocks * P > max_ctx_len), else
+ * HSWA_ERR_INVALID_ARG; a request whose ctx_len exceeds max_ctx_len is recorded as HSWA_ERR_BOUNDS. */
 hswa_status hswa_decode_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* q,
                              const void* k_new, const void* v_new, void* out, float* lse, void* workspace,
                              size_t workspace_bytes, void* stream);
@@ -162,7 +189,8 @@ hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* lay
  * and attends causally (to the cache and to new tokens 0..i; on SWA layers inside its own window).  The q_len
  * tokens end up appended (on a ring that requires q_len <= C - W + 1, checked: HSWA_ERR_INVALID_ARG): on Full
  * layers by an append launch ahead of one kernel that streams the KV once for all q_len tokens, on SWA layers
- * inside the attention kernel, which stages a ring once and gives every token its own warp.  Workspace: as
+ * inside the attention kernel, which stages a ring once and gives every token its own warp (that needs the
+ * whole ring in three 64-slot buffers: C > 192 with q_len > 1 is HSWA_ERR_UNSUPPORTED).  Workspace: as
  * hswa_decode_attn with max_total_q = max_batch * q_len.
  * After the step call hswa_step_advance with a q_indptr describing the ACCEPTED tokens per request. */
 hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, int32_t q_len,
@@ -191,15 +219,20 @@ hswa_status hswa_decode_attn_static_ws(hswa_handle* h, const hswa_layer* layer, 
                                        const void* q, const void* k_new, const void* v_new, void* out, float* lse,
                                        void* stream);
 
-/* Chunked prefill attention: request r extends its cached context by n[r] new tokens.
+/* Chunked prefill attention: request r extends its cached context by n[r] new tokens.  Paper Sec. 2.1:
+ * prefill is compute-bound; a Full layer attends the whole prefix plus the chunk causally, an SWA layer only
+ * inside its window of W keys, which is where the roughly 1/7 cost of the hybrid stack comes from; Sec. 5.2:
+ * fixed-size chunks against a growing cached prefix.
  * q: device bf16 [T][Hq][D]; k_new, v_new: device bf16 [T][Hkv][D] (required); out: device [T][Hq][D];
  * lse: device fp32 [T][Hq] or NULL.
  * Keys j < ctx[r] are read from the cache AS IT IS BEFORE THIS CHUNK'S APPEND (pages on a Full layer; the
  * ring on an SWA layer), keys j >= ctx[r] from k_new / v_new.  Causal mask on Full layers, causal + window
  * mask on SWA layers; key tiles wholly outside the mask are skipped.
- * fuse_append != 0: the chunk's K/V are also appended to the cache, ordered after every read of the old
- * ring contents (an SWA chunk longer than C - W + 1 tokens overwrites ring slots its own first queries
- * need, so "append, then attend" is not available on SWA layers). */
+ * fuse_append != 0: the chunk's K/V are also appended to the cache by a second launch (the append kernel of
+ * hswa_kv_append) queued on `stream` right behind the attention kernels, i.e. ordered after every read of the
+ * old ring contents (an SWA chunk longer than C - W + 1 tokens overwrites ring slots its own first queries
+ * need, so "append, then attend" is not available on SWA layers).  The append is fused into the call, not into
+ * the attention kernel. */
 hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* q,
                               const void* k_new, const void* v_new, int32_t fuse_append, void* out, float* lse,
                               void* workspace, size_t workspace_bytes, void* stream);
@@ -227,8 +260,9 @@ hswa_status hswa_swa_window_gather(hswa_handle* h, const hswa_layer* layer, cons
 hswa_status hswa_swa_window_scatter(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* buf,
                                     void* stream);
 
-/* Step advance, once per step after all layers: ctx_len[r] += n[r], ring_head[r] = (ring_head[r] + n[r])
- * mod C.  ctx_len, ring_head: device int32 [B], updated in place.  q_indptr: device or NULL (n = 1). */
+/* Step advance, once per step after all layers (paper Sec. 3.1.1: one logical view over both pools -- every
+ * layer of a step maps positions with the same lengths and ring heads, so they move once, after the last
+ * layer): ctx_len[r] += n[r], ring_head[r] = (ring_head[r] + n[r]) mod C.  ctx_len, ring_head: device int32 [B], updated in place.  q_indptr: device or NULL (n = 1). */
 hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
                               const int32_t* q_indptr, void* stream);
 
@@ -237,6 +271,14 @@ hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, i
 hswa_status hswa_get_async_error(hswa_handle* h, void* stream, int32_t info[4]);
 
 const char* hswa_status_string(hswa_status s);
+
+/* Self-test of the bounded waits (no paper counterpart; failure detection of the library itself).  Every wait
+ * on a pipeline barrier inside the kernels gives up after a fixed number of SM clocks, records
+ * HSWA_ERR_TIMEOUT in the error word and lets the block finish.  This call launches a one-block kernel whose
+ * consumer warp waits, with a limit of limit_clocks (1 .. 2e9), on a barrier that its producer never arms: the
+ * wait runs out, the kernel returns normally, and hswa_get_async_error then reports {HSWA_ERR_TIMEOUT, -1, 0, 7}.
+ * Nothing traps, nothing is left in flight, and the context stays usable. */
+hswa_status hswa_selftest_wait_timeout(hswa_handle* h, int64_t limit_clocks, void* stream);
 
 #ifdef __cplusplus
 }

@@ -29,6 +29,51 @@ def decode_algorithmic_bytes(w: Workload) -> int:
     return total
 
 
+def decode_unique_bytes(w: Workload) -> int:
+    """Like decode_algorithmic_bytes, but the KV of a prefix whose pages all requests share (paper Sec. 3.1.3:
+    equal prefixes share physical pages) is counted once per Full layer instead of once per request: the bytes a
+    sharing-aware kernel has to bring from HBM.  SWA layers hold private rings, so nothing is shared there."""
+    d, t = w.dims, w.tables
+    shared = t.shared_prefix_pages * d.page_size
+    total = 0
+    per_req_io = (2 * d.num_q_heads * d.head_dim * 2) + d.kv_bytes_per_token
+    for is_swa in w.layer_is_swa:
+        keys = int(attended_keys(is_swa, t.ctx_len, d.window).sum())
+        if not is_swa and t.batch > 0:
+            keys -= (t.batch - 1) * shared
+        total += keys * d.kv_bytes_per_token + t.batch * per_req_io
+    return total
+
+
+def decode_layer_bytes(w: Workload, is_swa: bool, unique: bool = False) -> int:
+    """Algorithmic bytes of one layer of the given kind in one decode step (logical, or with the shared prefix
+    counted once)."""
+    d, t = w.dims, w.tables
+    keys = int(attended_keys(is_swa, t.ctx_len, d.window).sum())
+    if unique and not is_swa and t.batch > 0:
+        keys -= (t.batch - 1) * t.shared_prefix_pages * d.page_size
+    return keys * d.kv_bytes_per_token + t.batch * ((2 * d.num_q_heads * d.head_dim * 2) + d.kv_bytes_per_token)
+
+
+def prefill_compulsory_bytes(w: Workload, is_swa: bool) -> int:
+    """Bytes one prefill layer must move: Q read, output written (bf16), the chunk's K/V read once, the cached keys
+    the chunk can see read once (Full: the whole context; SWA: at most W - 1 ring positions), and the appended K/V
+    written (SWA: the last min(n, C) tokens)."""
+    d, t = w.dims, w.tables
+    T = int(t.q_len.astype(np.int64).sum())
+    qo = 2 * T * d.num_q_heads * d.head_dim * 2
+    chunk_kv = T * d.kv_bytes_per_token
+    ctx = t.ctx_len.astype(np.int64)
+    n = t.q_len.astype(np.int64)
+    if is_swa:
+        cached = int(np.minimum(ctx, d.window - 1)[n > 0].sum())
+        written = int(np.minimum(n, d.ring_slots).sum())
+    else:
+        cached = int(ctx[n > 0].sum())
+        written = T
+    return qo + chunk_kv + (cached + written) * d.kv_bytes_per_token
+
+
 def prefill_pairs_per_head(w: Workload, is_swa: bool) -> int:
     """Unmasked (query, key) pairs per query head over the whole batch for one layer."""
     d, t = w.dims, w.tables

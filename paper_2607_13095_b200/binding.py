@@ -26,6 +26,7 @@ EXPORTS = [
     "hswa_create", "hswa_destroy", "hswa_workspace_bytes", "hswa_validate_batch", "hswa_kv_append",
     "hswa_decode_attn", "hswa_decode_attn_mtp", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
     "hswa_window_safe_len", "hswa_swa_window_gather", "hswa_swa_window_scatter",
+    "hswa_decode_workspace_need", "hswa_selftest_wait_timeout", "hswa_set_overlap",
 ]
 
 
@@ -78,6 +79,12 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_destroy.argtypes = [vp]
     lib.hswa_workspace_bytes.restype = sz
     lib.hswa_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    lib.hswa_decode_workspace_need.restype = sz
+    lib.hswa_decode_workspace_need.argtypes = [vp, i32, i32, i32, i32, i32]
+    lib.hswa_set_overlap.restype = C.c_int
+    lib.hswa_set_overlap.argtypes = [vp, i32]
+    lib.hswa_selftest_wait_timeout.restype = C.c_int
+    lib.hswa_selftest_wait_timeout.argtypes = [vp, i64, vp]
     lib.hswa_validate_batch.restype = C.c_int
     lib.hswa_validate_batch.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp]
     lib.hswa_kv_append.restype = C.c_int
@@ -189,6 +196,19 @@ class Batch:
 
 def hswa_workspace_bytes(h: Handle, max_batch: int, max_total_q: int, max_ctx_len: int) -> int:
     return int(load().hswa_workspace_bytes(h.ptr, max_batch, max_total_q, max_ctx_len))
+
+
+def hswa_decode_workspace_need(h: Handle, is_swa: bool, batch: int, max_ctx_len: int, shared_prefix_len: int = 0,
+                               q_len: int = 1) -> int:
+    return int(load().hswa_decode_workspace_need(h.ptr, int(bool(is_swa)), batch, max_ctx_len, shared_prefix_len, q_len))
+
+
+def hswa_set_overlap(h: Handle, enabled: bool):
+    _check(load().hswa_set_overlap(h.ptr, int(bool(enabled))), "hswa_set_overlap")
+
+
+def hswa_selftest_wait_timeout(h: Handle, limit_clocks: int):
+    _check(load().hswa_selftest_wait_timeout(h.ptr, int(limit_clocks), _stream()), "hswa_selftest_wait_timeout")
 
 
 def hswa_validate_batch(h: Handle, layer: Layer, batch: Batch):

@@ -73,6 +73,51 @@ int plan_max_splits(int split_len, int max_ctx_len) {
   return (int)((kv_len + split_len - 1) / split_len);
 }
 
+// Everything the host decides about one decode call from host-known values only (so that results do not depend
+// on where pages sit): whether the shared-prefix stage runs and in how many slices, the split length of the
+// streaming kernel, the partial slots per (request, token, head) row and the scratch bytes they take.
+struct DecodePlan {
+  bool cascade;
+  int prefix_slices, prefix_tps;  // shared-prefix stage: slices and 128-key tiles per slice
+  int k_start, split_base;        // first key and first partial slot of the streaming kernel
+  int split_len, grid_splits, max_splits;
+  size_t o_bytes, ml_bytes;       // scratch: o partials, then (m, l) pairs; 0 when rows are written directly
+};
+
+bool plan_decode(const hswa_handle* h, int is_swa, int batch, int max_ctx_len, int shared_prefix_len, int q_len,
+                 DecodePlan* pl) {
+  DecodePlan d = {};
+  d.cascade = !is_swa && q_len == 1 && shared_prefix_len >= 128 && h->cfg.head_dim == 128 && h->cfg.page_size == 64 &&
+              h->group == 8;
+  if (is_swa) {
+    d.split_len = ((h->ring_slots + 63) / 64) * 64;
+    d.grid_splits = d.max_splits = 1;
+  } else {
+    if (d.cascade) {
+      const int tiles = (shared_prefix_len + 127) / 128;
+      const int base = ((batch + 31) / 32) * h->cfg.num_kv_heads;
+      int want = h->num_sms / base;
+      want = want < 1 ? 1 : (want > tiles ? tiles : want);
+      d.prefix_tps = (tiles + want - 1) / want;
+      d.prefix_slices = (tiles + d.prefix_tps - 1) / d.prefix_tps;  // no slice is empty
+      d.k_start = shared_prefix_len;
+      d.split_base = d.prefix_slices;
+    }
+    const int last = max_ctx_len + q_len - 1 - d.k_start;  // highest key position the streaming kernel covers, relative
+    d.split_len = plan_split_len(h, batch, last);
+    d.grid_splits = plan_max_splits(d.split_len, last);
+    d.max_splits = d.split_base + d.grid_splits;
+    if (d.grid_splits > 65535) return false;
+    if (d.max_splits > 1) {
+      const size_t rows = (size_t)batch * q_len * h->cfg.num_q_heads;
+      d.o_bytes = (rows * d.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
+      d.ml_bytes = (rows * d.max_splits * sizeof(float2) + 255) & ~size_t(255);
+    }
+  }
+  *pl = d;
+  return true;
+}
+
 // 4-D view of a pool for TMA: {D, P, 2 * Hkv, num_pages}, box {64, box_slots, 1, 1} (0: a whole page),
 // 128-byte swizzle.
 hswa_status make_pool_map(const hswa_handle* h, const hswa_layer* layer, CUtensorMap* tm, int box_slots = 0) {
@@ -154,7 +199,9 @@ hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out) {
   h->encode_tiled = nullptr;
   h->chain_stream = nullptr;
   h->chain_ctx = nullptr;
+  h->chain_pool = nullptr;
   h->chain_ok = 0;
+  h->overlap_enabled = 1;
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -199,13 +246,36 @@ size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max
   return ((o_bytes + 255) & ~size_t(255)) + ((ml_bytes + 255) & ~size_t(255));
 }
 
+size_t hswa_decode_workspace_need(const hswa_handle* h, int32_t is_swa, int32_t batch, int32_t max_ctx_len,
+                                  int32_t shared_prefix_len, int32_t q_len) {
+  if (!h || batch <= 0 || max_ctx_len < 0 || shared_prefix_len < 0 || shared_prefix_len > max_ctx_len || q_len < 1 || q_len > 4)
+    return 0;
+  DecodePlan pl;
+  if (!plan_decode(h, is_swa, batch, max_ctx_len, shared_prefix_len, q_len, &pl)) return 0;
+  return pl.o_bytes + pl.ml_bytes;
+}
+
+hswa_status hswa_set_overlap(hswa_handle* h, int32_t enabled) {
+  if (!h) return HSWA_ERR_INVALID_ARG;
+  h->overlap_enabled = enabled != 0;
+  h->chain_ok = 0;
+  return HSWA_OK;
+}
+
+hswa_status hswa_selftest_wait_timeout(hswa_handle* h, int64_t limit_clocks, void* stream) {
+  if (!h || limit_clocks < 1 || limit_clocks > 2000000000LL) return HSWA_ERR_INVALID_ARG;
+  h->chain_ok = 0;
+  if (cudaSetDevice(h->device) != cudaSuccess) return HSWA_ERR_CUDA;
+  return hswa_launch_wait_selftest(limit_clocks, h->err, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
 hswa_status hswa_validate_batch(hswa_handle* h, const hswa_layer* layer, const hswa_batch* b, void* stream) {
   if (h) h->chain_ok = 0;
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
   if (cudaSetDevice(h->device) != cudaSuccess) return HSWA_ERR_CUDA;
-  cudaError_t e = hswa_launch_validate(model_params(h), batch_params(b), layer->is_swa, layer->num_pages, h->err,
-                                       (cudaStream_t)stream);
+  cudaError_t e = hswa_launch_validate(model_params(h), batch_params(b), layer->is_swa, layer->num_pages, b->max_ctx_len,
+                                       b->max_q_len, h->err, (cudaStream_t)stream);
   return e == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
@@ -227,6 +297,7 @@ hswa_status hswa_kv_append(hswa_handle* h, const hswa_layer* layer, const hswa_b
   p.total_q = b->total_q;
   p.max_q_len = b->max_q_len;
   p.uniform_n = 0;
+  p.err = h->err;
   return hswa_launch_append(p, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
 }
 
@@ -240,6 +311,8 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
   if (!q || !out || !aligned16(q) || !aligned16(out)) return HSWA_ERR_INVALID_ARG;
   if ((k_new == nullptr) != (v_new == nullptr)) return HSWA_ERR_INVALID_ARG;
   if (k_new && (!aligned16(k_new) || !aligned16(v_new))) return HSWA_ERR_INVALID_ARG;
+  // the block table must cover every position the host bound allows (position max_ctx_len is the new token's)
+  if (!layer->is_swa && (int64_t)b->max_ctx_len + 1 > (int64_t)b->max_blocks * h->cfg.page_size) return HSWA_ERR_INVALID_ARG;
 
   DecodeParams p;
   p.m = model_params(h);
@@ -258,40 +331,23 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
   p.k_start = 0;
   p.split_base = 0;
   p.nq = 1;
+  p.max_ctx_len = b->max_ctx_len;
   // Cascade decode: the shared prefix is attended once per group of requests on the tensor cores, the
   // per-request suffixes by the streaming kernel; both leave partials for the combine.
-  const bool cascade = !layer->is_swa && shared_prefix_len >= 128 && h->cfg.head_dim == 128 && h->cfg.page_size == 64 &&
-                       h->group == 8;
-  int prefix_slices = 0, prefix_tps = 0;
-  if (layer->is_swa) {
-    p.split_len = ((h->ring_slots + 63) / 64) * 64;
-    p.max_splits = 1;
-    p.grid_splits = 1;
-  } else {
-    if (cascade) {
-      const int tiles = (shared_prefix_len + 127) / 128;
-      const int base = ((b->batch + 31) / 32) * h->cfg.num_kv_heads;
-      int want = h->num_sms / base;
-      want = want < 1 ? 1 : (want > tiles ? tiles : want);
-      prefix_tps = (tiles + want - 1) / want;
-      prefix_slices = (tiles + prefix_tps - 1) / prefix_tps;  // no slice is empty
-      p.k_start = shared_prefix_len;
-      p.split_base = prefix_slices;
-    }
-    const int suffix_ctx = b->max_ctx_len - p.k_start;  // longest key range the streaming kernel covers, minus one
-    p.split_len = plan_split_len(h, b->batch, suffix_ctx);
-    p.grid_splits = plan_max_splits(p.split_len, suffix_ctx);
-    p.max_splits = p.split_base + p.grid_splits;
-    if (p.grid_splits > 65535) return HSWA_ERR_UNSUPPORTED;
-    if (p.max_splits > 1) {
-      const size_t rows = (size_t)b->batch * h->cfg.num_q_heads;
-      const size_t o_bytes = (rows * p.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
-      const size_t ml_bytes = (rows * p.max_splits * sizeof(float2) + 255) & ~size_t(255);
-      if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < o_bytes + ml_bytes)
-        return HSWA_ERR_WORKSPACE;
-      p.part_o = static_cast<float*>(workspace);
-      p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + o_bytes);
-    }
+  DecodePlan pl;
+  if (!plan_decode(h, layer->is_swa, b->batch, b->max_ctx_len, shared_prefix_len, 1, &pl)) return HSWA_ERR_UNSUPPORTED;
+  const bool cascade = pl.cascade;
+  const int prefix_slices = pl.prefix_slices, prefix_tps = pl.prefix_tps;
+  p.k_start = pl.k_start;
+  p.split_base = pl.split_base;
+  p.split_len = pl.split_len;
+  p.grid_splits = pl.grid_splits;
+  p.max_splits = pl.max_splits;
+  if (p.max_splits > 1) {
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < pl.o_bytes + pl.ml_bytes)
+      return HSWA_ERR_WORKSPACE;
+    p.part_o = static_cast<float*>(workspace);
+    p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + pl.o_bytes);
   }
   CUtensorMap tm;
   // SWA layers: the ring kernel loads 16-slot granules, only those that meet the window
@@ -299,7 +355,9 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
   if (st != HSWA_OK) return st;
   // A fused decode that directly follows another fused decode of the same step (same handle, stream and batch
   // arrays) may start early: those kernels never write the batch arrays or another layer's pool.
-  const bool early = h->chain_ok && k_new != nullptr && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len;
+  // The previous kernel appends to its own layer's pool, so a call on that same pool waits for it to finish.
+  const bool early = h->overlap_enabled && h->chain_ok && k_new != nullptr && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len &&
+                     h->chain_pool != (const void*)layer->pool;
   h->chain_ok = 0;
   if (cascade) {
     PrefillParams pp = {};
@@ -326,6 +384,7 @@ static hswa_status decode_impl(hswa_handle* h, const hswa_layer* layer, const hs
     h->chain_ok = 1;
     h->chain_stream = stream;
     h->chain_ctx = (const void*)b->ctx_len;
+    h->chain_pool = (const void*)layer->pool;
   }
   return HSWA_OK;
 }
@@ -343,13 +402,17 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   hswa_status st = check_common(h, layer, b);
   if (st != HSWA_OK) return st;
   // a ring kernel with the append fused may start early behind another fused decode kernel of the same step
-  const bool early = layer->is_swa && h->chain_ok && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len;
+  const bool early = h->overlap_enabled && layer->is_swa && h->chain_ok && h->chain_stream == stream && h->chain_ctx == (const void*)b->ctx_len &&
+                     h->chain_pool != (const void*)layer->pool;
   h->chain_ok = 0;
   if (b->q_indptr != nullptr || q_len < 1 || q_len > 4) return HSWA_ERR_INVALID_ARG;
   if (b->batch == 0) return HSWA_OK;
   if (!q || !out || !k_new || !v_new) return HSWA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return HSWA_ERR_INVALID_ARG;
   if (layer->is_swa && q_len > h->ring_slots - h->cfg.window + 1) return HSWA_ERR_INVALID_ARG;  // append-then-attend limit
+  // the token mode of the ring kernel keeps a whole ring staged (three 64-slot buffers) while its warps patch and read it
+  if (layer->is_swa && (h->ring_slots + 63) / 64 > 3) return HSWA_ERR_UNSUPPORTED;
+  if (!layer->is_swa && (int64_t)b->max_ctx_len + q_len > (int64_t)b->max_blocks * h->cfg.page_size) return HSWA_ERR_INVALID_ARG;
 
   AppendParams a;
   a.m = model_params(h);
@@ -362,6 +425,7 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   a.total_q = b->batch * q_len;
   a.max_q_len = q_len;
   a.uniform_n = q_len;
+  a.err = h->err;
 
   DecodeParams p;
   p.m = a.m;
@@ -382,24 +446,17 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   p.k_start = 0;
   p.split_base = 0;
   p.nq = q_len;
-  if (layer->is_swa) {
-    p.split_len = ((h->ring_slots + 63) / 64) * 64;
-    p.grid_splits = 1;
-  } else {
-    const int last = b->max_ctx_len + q_len - 1;  // highest key position
-    p.split_len = plan_split_len(h, b->batch, last);
-    p.grid_splits = plan_max_splits(p.split_len, last);
-    if (p.grid_splits > 65535) return HSWA_ERR_UNSUPPORTED;
-  }
-  p.max_splits = p.grid_splits;
+  p.max_ctx_len = b->max_ctx_len;
+  DecodePlan pl;
+  if (!plan_decode(h, layer->is_swa, b->batch, b->max_ctx_len, 0, q_len, &pl)) return HSWA_ERR_UNSUPPORTED;
+  p.split_len = pl.split_len;
+  p.grid_splits = pl.grid_splits;
+  p.max_splits = pl.max_splits;
   if (p.max_splits > 1) {
-    const size_t rows = (size_t)b->batch * q_len * h->cfg.num_q_heads;
-    const size_t o_bytes = (rows * p.max_splits * h->cfg.head_dim * sizeof(float) + 255) & ~size_t(255);
-    const size_t ml_bytes = (rows * p.max_splits * sizeof(float2) + 255) & ~size_t(255);
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < o_bytes + ml_bytes)
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < pl.o_bytes + pl.ml_bytes)
       return HSWA_ERR_WORKSPACE;
     p.part_o = static_cast<float*>(workspace);
-    p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + o_bytes);
+    p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + pl.o_bytes);
   }
   CUtensorMap tm;
   const int granule = h->cfg.page_size < HSWA_RING_GRANULE ? h->cfg.page_size : HSWA_RING_GRANULE;
@@ -410,6 +467,7 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   h->chain_ok = 1;  // none of these kernels writes the batch arrays or another layer's pool
   h->chain_stream = stream;
   h->chain_ctx = (const void*)b->ctx_len;
+  h->chain_pool = (const void*)layer->pool;
   return HSWA_OK;
 }
 
@@ -495,6 +553,7 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
     a.total_q = p.total_q;
     a.max_q_len = p.max_q_len;
     a.uniform_n = 0;
+    a.err = h->err;
     if (hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
   }
   return HSWA_OK;

@@ -30,10 +30,16 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
   const int t0 = p.uniform_n > 0 ? r * p.uniform_n : (p.b.q_indptr ? p.b.q_indptr[r] : r);
   const int pos = p.b.ctx_len[r] + (t - t0);
   const int blk = pos / M.P;
-  if (blk >= p.b.max_blocks) return;
+  if (pos < 0 || blk >= p.b.max_blocks) {  // the block table does not cover this position: skip the write
+    if (lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -3, blk);
+    return;
+  }
   const int page = p.b.block_table[(int64_t)r * p.b.max_blocks + blk];
   const int slot = pos % M.P;
-  if (page < 0 || page >= p.num_pages) return;
+  if (page < 0 || page >= p.num_pages) {
+    if (lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, blk, page);
+    return;
+  }
   const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + (int64_t)t * M.Hkv * M.D;
   __nv_bfloat16* dst = p.pool + (((int64_t)page * 2 + kv) * M.Hkv * M.P + slot) * M.D;  // head 0 of this (page, K|V)
   for (int c0 = lane; c0 < chunks; c0 += 128) {
@@ -75,7 +81,10 @@ __global__ void __launch_bounds__(256) append_ring_kernel(const AppendParams p) 
   const int s = math_mod(p.b.ring_head[r] + (i % M.C), M.C);
   const int page = p.b.ring_table[(int64_t)r * M.R + s / M.P];
   const int slot = s % M.P;
-  if (page < 0 || page >= p.num_pages) return;
+  if (page < 0 || page >= p.num_pages) {
+    record_error(p.err, HSWA_ERR_BOUNDS, r, s / M.P, page);
+    return;
+  }
   const __nv_bfloat16* src = (kv == 0 ? p.k_new : p.v_new) + ((int64_t)(t0 + i) * M.Hkv + kh) * M.D + ch * 8;
   __nv_bfloat16* dst = p.pool + ((((int64_t)page * 2 + kv) * M.Hkv + kh) * M.P + slot) * M.D + ch * 8;
   *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
@@ -130,13 +139,14 @@ __global__ void advance_kernel(ModelParams M, int B, int32_t* ctx_len, int32_t* 
 
 // One block per request; threads scan the table entries the step would touch.
 __global__ void __launch_bounds__(128) validate_kernel(ModelParams M, BatchParams b, int is_swa, int64_t num_pages,
-                                                       int32_t* err) {
+                                                       int max_ctx_len, int max_q_len, int32_t* err) {
   const int r = blockIdx.x;
   const int ctx = b.ctx_len[r];
   const int n = b.q_indptr ? b.q_indptr[r + 1] - b.q_indptr[r] : 1;
   if (threadIdx.x == 0) {
-    if (ctx < 0) record_error(err, HSWA_ERR_BOUNDS, r, -1, ctx);
-    if (n < 0) record_error(err, HSWA_ERR_BOUNDS, r, -2, n);
+    // the launch geometry of every kernel is planned from the host's bounds: a longer request would lose keys
+    if (ctx < 0 || ctx > max_ctx_len) record_error(err, HSWA_ERR_BOUNDS, r, -1, ctx);
+    if (n < 0 || n > max_q_len) record_error(err, HSWA_ERR_BOUNDS, r, -2, n);
   }
   if (ctx < 0 || n < 0) return;
   if (!is_swa) {
@@ -158,6 +168,23 @@ __global__ void __launch_bounds__(128) validate_kernel(ModelParams M, BatchParam
       const int pg = b.ring_table[(int64_t)r * M.R + i];
       if (pg < 0 || pg >= num_pages) record_error(err, HSWA_ERR_BOUNDS, r, i, pg);
     }
+  }
+}
+
+// Self-test of the bounded-wait path every pipeline kernel relies on: warp 1 waits, with the given limit, on an
+// mbarrier that warp 0 (the would-be producer) never arms.  The wait runs out, the waiter records
+// HSWA_ERR_TIMEOUT in the error word exactly as the pipeline kernels do, and the block returns normally:
+// nothing spins past the limit and nothing is left in flight.
+__global__ void __launch_bounds__(64) wait_selftest_kernel(long long limit_clocks, int32_t* err) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) {
+    const bool ok = mbar_wait(smem_u32(&bar), 0, limit_clocks);
+    if (!ok && (threadIdx.x & 31) == 0) record_error(err, HSWA_ERR_TIMEOUT, -1, 0, 7);
   }
 }
 
@@ -186,9 +213,14 @@ cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_le
 }
 
 cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
-                                 int32_t* err, cudaStream_t s) {
+                                 int32_t max_ctx_len, int32_t max_q_len, int32_t* err, cudaStream_t s) {
   if (b.B == 0) return cudaSuccess;
-  validate_kernel<<<b.B, 128, 0, s>>>(m, b, is_swa, num_pages, err);
+  validate_kernel<<<b.B, 128, 0, s>>>(m, b, is_swa, num_pages, max_ctx_len, max_q_len, err);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_wait_selftest(int64_t limit_clocks, int32_t* err, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 64, 0, s>>>((long long)limit_clocks, err);
   return cudaGetLastError();
 }
 

@@ -187,6 +187,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
   const ModelParams& M = p.m;
   const int ctx = p.b.ctx_len[r];
   const int kv_len = ctx + 1;
+  // the grid was sized from the host's bound: a longer context would silently lose its tail
+  if (threadIdx.x == 0 && split == 0 && kh == 0 && ctx > p.max_ctx_len) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, ctx);
 
   KeyRange kr;
   kr.is_swa = p.is_swa;
@@ -500,6 +502,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * NS];
+  __shared__ int s_abort;  // token mode: a warp's wait ran out; all token warps leave together at the next barrier
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
   float* sc_o = reinterpret_cast<float*>(smem + NS * STAGE_BYTES);  // [NW][8][D]
@@ -523,6 +526,7 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
     }
     mbar_fence_init();
     tma_prefetch_desc(&tm_pool);
+    s_abort = 0;
   }
   __syncthreads();
 
@@ -663,8 +667,10 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
           if (!mbar_wait(smem_u32(&bars[g % NS]), (g / NS) & 1)) {
             if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
             ok = false;
+            break;
           }
         }
+        if (!ok && lane == 0) *reinterpret_cast<volatile int*>(&s_abort) = 1;
         if (fuse && ok) {
           const int t_new = kr.head / TK, row = kr.head % TK;
           uint8_t* sK = smem + ((k * n_tiles + t_new) % NS) * STAGE_BYTES;
@@ -680,7 +686,8 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
           }
           fence_proxy_async_smem();
         }
-        if (fuse) asm volatile("bar.sync 1, %0;" ::"r"(nq * 32) : "memory");  // all nq rows are in the tiles now
+        asm volatile("bar.sync 1, %0;" ::"r"(nq * 32) : "memory");  // all nq rows are in the tiles now
+        if (*reinterpret_cast<volatile int*>(&s_abort)) break;  // same value in every token warp: they stop together
         float m_run[2] = {-INFINITY, -INFINITY};
         float l_run[2] = {0.f, 0.f};
         float o[KS][4];
@@ -946,6 +953,7 @@ decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParam
   const int nq = p.nq;
   const int ctx = p.b.ctx_len[r];
   const int kv_len = ctx + nq;
+  if (threadIdx.x == 0 && split == 0 && kh == 0 && ctx > p.max_ctx_len) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, ctx);
 
   KeyRangeMulti kr;
   kr.ctx = ctx;

@@ -26,7 +26,9 @@ struct hswa_handle {
   // the next fused decode may overlap its prologue and cache loads with that kernel's tail.
   void* chain_stream;
   const void* chain_ctx;
+  const void* chain_pool;  // pool of the previous fused decode: a kernel must not start early on the pool its predecessor writes
   int32_t chain_ok;
+  int32_t overlap_enabled;  // hswa_set_overlap
 };
 
 // Model constants every kernel needs.
@@ -64,6 +66,7 @@ struct DecodeParams {
   int32_t split_base;  // partial slot of this launch's split 0
   int32_t grid_splits; // splits this launch covers (grid extent)
   int32_t nq;          // new tokens per request (1; 2-4 for multi-token decode)
+  int32_t max_ctx_len; // host-known bound of ctx_len the launch geometry was planned for
   float* part_o;       // [B*Hq][max_splits][D]
   float2* part_ml;     // [B*Hq][max_splits] (m in log2 units, l)
   int32_t* err;
@@ -80,6 +83,7 @@ struct AppendParams {
   int32_t total_q;
   int32_t max_q_len;  // host-known bound of new tokens per request
   int32_t uniform_n;  // > 0: every request has exactly this many new tokens and q_indptr is ignored
+  int32_t* err;       // device error word: out-of-range block index or page id is recorded, the write skipped
 };
 
 struct PrefillParams {
@@ -130,7 +134,8 @@ cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_le
 cudaError_t hswa_launch_window_move(const ModelParams& m, const BatchParams& b, __nv_bfloat16* pool, int64_t num_pages,
                                     __nv_bfloat16* buf, int gather, int32_t* err, cudaStream_t s);
 cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
-                                 int32_t* err, cudaStream_t s);
+                                 int32_t max_ctx_len, int32_t max_q_len, int32_t* err, cudaStream_t s);
+cudaError_t hswa_launch_wait_selftest(int64_t limit_clocks, int32_t* err, cudaStream_t s);
 
 #ifdef __CUDACC__
 namespace hswa_dev {
@@ -169,15 +174,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after about two seconds of SM clocks and reports false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after `limit` SM clocks (default: about two seconds) and reports false.
+constexpr long long kWaitLimitClocks = 4000000000LL;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitLimitClocks) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > 4000000000LL) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -118,3 +118,40 @@ def test_config3_chunked_prefill_fullsize():
         assert (err <= bound).all(), ("swa" if is_swa else "full", float(err.max()))
         orc.kv_append(cfg, layer, ob, k, v)
         assert np.array_equal(to_host_bits(pb.layers[i].pool), before), (i, "pool bytes after prefill append")
+
+
+def test_config5_seventy_layer_step_late_layers():
+    """The whole 70-layer step bench.py times (100 GB of pools, every layer's kernels chained on one stream), checked
+    on a late Full layer (63) and the SWA layer behind it (64): sampled output rows and the appended rows of a few
+    requests, whose pages are gathered on the device so that no 10 GB pool crosses to the host."""
+    dev = torch.device("cuda", 0)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 120e9:
+        pytest.skip("needs 120 GB of free device memory")
+    w = bench.make_workload("cfg5")
+    b = bench.DecodeBench(w, 4, dev)
+    t, d = b.t, w.dims
+    assert len(b.layers) == 70 and not w.layer_is_swa[63] and w.layer_is_swa[64]
+    cfg = orc.OracleConfig(d.num_q_heads, d.num_kv_heads, d.head_dim, d.page_size, d.window, d.ring_pages)
+    reqs = bench.pick_requests(t, 3)
+    bt, full_ids, rt, ring_ids = bench.compact_tables(t, d, reqs)
+    ridx = torch.from_numpy(reqs).to(dev)
+    gather = {63: torch.from_numpy(full_ids).to(dev), 64: torch.from_numpy(ring_ids).to(dev)}
+    before = {i: to_host_bits(b.layers[i].pool.index_select(0, gather[i])) for i in (63, 64)}
+    b.step()
+    torch.cuda.synchronize()
+    assert hb.hswa_get_async_error(b.h)[0] == hb.HSWA_OK
+    ob = orc.OracleBatch(t.ctx_len[reqs], bt, rt, t.ring_head[reqs])
+    rng = np.random.default_rng(7)
+    for i, heads in ((63, rng.choice(d.num_q_heads, 12, replace=False)), (64, np.arange(d.num_q_heads))):
+        is_swa = w.layer_is_swa[i]
+        tok = np.repeat(np.arange(len(reqs)), len(heads)).astype(np.int32)
+        head = np.tile(heads, len(reqs)).astype(np.int32)
+        q, k, v = (to_host_bits(x[i].index_select(0, ridx)) for x in (b.q, b.k_new, b.v_new))
+        layer = orc.OracleLayer(before[i], is_swa)
+        ref, _ = orc.attention(cfg, layer, ob, q, k, v, rows=(tok, head))
+        got = b.out[i].index_select(0, ridx).float().cpu().numpy()[tok, head]
+        assert np.abs(got - ref).max() <= TOL, (i, float(np.abs(got - ref).max()))
+        orc.kv_append(cfg, layer, ob, k, v)
+        after = to_host_bits(b.layers[i].pool.index_select(0, gather[i]))
+        assert np.array_equal(after, before[i]), (i, "pool bytes after the fused append")

@@ -325,3 +325,33 @@ def test_step_advance_and_mod():
     b = orc.OracleBatch(np.array([10], np.int32), np.zeros((1, 4), np.int32), np.array([[7, 8, 9]], np.int32),
                         np.array([1], np.int32))
     assert orc.locate(cfg, True, b, 0, 8) == (9, 3)   # slot (1 - 2) mod 12 = 11 -> page index 2, slot 3
+
+
+def test_locate_hand_worked_literals():
+    """Position -> (page, slot) worked by hand from the two storage rules (Full: block p div P of the request's
+    table, slot p mod P; SWA: ring slot (head + p - ctx) mod C, page = ring_table[slot div P]), on permuted tables,
+    for both layer kinds, including wrapped rings and positions behind and ahead of the ring head."""
+    cfg = oracle_config(D8)                                    # W = 8, P = 4, R = 3, C = 12
+    bt = np.array([[1, 3, 7, 4], [5, 2, 9, 0]], np.int32)
+    rt = np.array([[7, 8, 9], [8, 2, 5]], np.int32)
+    b = orc.OracleBatch(np.array([10, 30], np.int32), bt, rt, np.array([1, 10], np.int32))
+    full = {(0, 6): (3, 2), (1, 0): (5, 0), (1, 3): (5, 3), (1, 4): (2, 0), (1, 11): (9, 3), (1, 13): (0, 1)}
+    for (r, p), want in full.items():
+        assert orc.locate(cfg, False, b, r, p) == want, (r, p)
+    swa = {
+        (0, 10): (7, 1),    # the next write sits at the ring head
+        (0, 9): (7, 0), (0, 8): (9, 3),     # one and two back: the second wraps to the last page
+        (0, 3): (8, 2),     # (1 - 7) mod 12 = 6
+        (0, 11): (7, 2), (0, 13): (8, 0),   # new tokens ahead of the head
+        (1, 30): (5, 2), (1, 31): (5, 3), (1, 32): (8, 0),   # head 10: the third new token wraps to slot 0
+        (1, 23): (8, 3),    # oldest key of a window of 8: (10 - 7) = 3
+        (1, 25): (2, 1), (1, 19): (5, 3),   # (10 - 11) mod 12 = 11
+    }
+    for (r, p), want in swa.items():
+        assert orc.locate(cfg, True, b, r, p) == want, (r, p)
+    big = oracle_config(wl.BIG)                                # W = 128, P = 64, R = 3, C = 192
+    b = orc.OracleBatch(np.array([5000], np.int32), np.array([[11, 0, 6]], np.int32), np.array([[40, 3, 17]], np.int32),
+                        np.array([190], np.int32))
+    assert orc.locate(big, False, b, 0, 64) == (0, 0) and orc.locate(big, False, b, 0, 191) == (6, 63)
+    for p, want in {5000: (17, 62), 5001: (17, 63), 5002: (40, 0), 4873: (40, 63), 4936: (3, 62), 4999: (17, 61)}.items():
+        assert orc.locate(big, True, b, 0, p) == want, p
