@@ -260,6 +260,33 @@ hswa_status hswa_swa_window_gather(hswa_handle* h, const hswa_layer* layer, cons
 hswa_status hswa_swa_window_scatter(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, const void* buf,
                                     void* stream);
 
+/* Out-of-window SWA release bookkeeping and dual-index matching (paper Sec. 3.1.3 items 2 and 3).
+ *
+ * State: swa_valid_from[r] (device int32 [B], caller-owned, starts at 0 for a fresh request, or at
+ * max(0, ctx - (W - 1)) for a ring seeded with hswa_swa_window_scatter) is the first cached position of request
+ * r whose SWA KV is still valid; the valid SWA positions of a live request are the suffix [swa_valid_from, ctx).
+ *
+ * hswa_swa_release, once per step AFTER hswa_step_advance: moves the boundary forward to ctx - C (the ring has
+ * overwritten everything older) and, for requests with release[r] != 0 (device uint8 [B]; NULL: all), to
+ * ctx - (W - 1): the paper's release events -- a prefill chunk completed, the request terminated, every N tokens
+ * generated in decode -- drop everything the next token's window cannot reach, which keeps SWA use at window
+ * magnitude.  Which event fired is the scheduler's knowledge, hence the flags.  The boundary never moves back.
+ *
+ * hswa_swa_valid_mask: the per-position SWA status a prefix-tree node records: mask[r][p] = 1 iff
+ * swa_valid_from[r] <= p < ctx_len[r], for p < mask_stride (0 beyond ctx); mask is uint8 [B][mask_stride] in
+ * device memory or pinned host memory.
+ *
+ * hswa_prefix_hit_len: pure host arithmetic.  A cached prefix matches a new request on its first match_len tokens;
+ * its nodes carry per-token Full status (full_valid, host uint8, NULL: nothing valid) and SWA status (swa_valid, as
+ * for hswa_window_safe_len).  Returns the largest L <= match_len such that every position in [0, L) has Full KV
+ * (Full layers read all of them) and every position in [max(0, L - (W - 1)), L) has SWA KV.  Evicting the SWA part
+ * of old segments on its own therefore keeps the prefix reusable; evicting a whole segment ends it there. */
+hswa_status hswa_swa_release(hswa_handle* h, int32_t batch, const int32_t* ctx_len, const uint8_t* release,
+                             int32_t* swa_valid_from, void* stream);
+hswa_status hswa_swa_valid_mask(hswa_handle* h, int32_t batch, const int32_t* ctx_len, const int32_t* swa_valid_from,
+                                int64_t mask_stride, uint8_t* mask, void* stream);
+int64_t hswa_prefix_hit_len(int64_t match_len, int32_t window, const uint8_t* full_valid, const uint8_t* swa_valid);
+
 /* Step advance, once per step after all layers (paper Sec. 3.1.1: one logical view over both pools -- every
  * layer of a step maps positions with the same lengths and ring heads, so they move once, after the last
  * layer): ctx_len[r] += n[r], ring_head[r] = (ring_head[r] + n[r]) mod C.  ctx_len, ring_head: device int32 [B], updated in place.  q_indptr: device or NULL (n = 1). */

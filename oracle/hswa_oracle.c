@@ -352,3 +352,65 @@ int orc_window_scatter(const orc_config* cfg, const orc_layer* L, const orc_batc
     }
   return ORC_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Out-of-window SWA release and dual-index matching (paper Sec. 3.1.3 items 2 and 3).
+ *
+ * State per live request: swa_valid_from[r], the first cached position whose SWA KV is still valid.  The valid
+ * SWA positions of a live request are always the suffix [swa_valid_from, len): KV is written in position order
+ * and only ever dropped from the old end.  Two things move the boundary forward:
+ *   storage   a ring of C slots holds the last C positions at most, later writes win (Sec. 3.1.1 "strictly
+ *             O(W)"): after any append, swa_valid_from >= len - C;
+ *   release   on the paper's three events -- a prefill chunk completes, the request terminates, every N tokens
+ *             generated during decode -- everything outside the window is released.  The next token, at position
+ *             len, reads the W - 1 cached positions [len - (W - 1), len) (the window includes the query itself),
+ *             so a release sets swa_valid_from >= len - (W - 1).
+ * ctx_len holds the lengths AFTER the step's advance; release[r] != 0 marks the requests whose event fired
+ * (NULL: all of them).  The boundary never moves back and never goes below 0. */
+int orc_swa_release(const orc_config* cfg, int32_t batch, const int32_t* ctx_len, const uint8_t* release,
+                    int32_t* swa_valid_from) {
+  const int64_t C = (int64_t)cfg->ring_pages * cfg->page_size;
+  const int64_t W = cfg->window;
+  for (int32_t r = 0; r < batch; ++r) {
+    int64_t from = swa_valid_from[r];
+    const int64_t len = ctx_len[r];
+    if (len - C > from) from = len - C;                                  /* overwritten by the ring */
+    if ((release == NULL || release[r]) && len - (W - 1) > from) from = len - (W - 1); /* released */
+    if (from < 0) from = 0;
+    swa_valid_from[r] = (int32_t)from;
+  }
+  return ORC_OK;
+}
+
+/* Does a release fire?  kind 0: a prefill chunk has completed; kind 1: the request has terminated; kind 2: a
+ * token has been generated in decode, `decoded` tokens so far including this one, release every every_n. */
+int orc_release_due(int32_t kind, int64_t decoded, int64_t every_n) {
+  if (kind == 0 || kind == 1) return 1;
+  if (kind == 2) return every_n > 0 && decoded > 0 && decoded % every_n == 0;
+  return 0;
+}
+
+/* Per-position SWA status of a request of length len: mask[p] = 1 iff swa_valid_from <= p < len. */
+int orc_swa_valid_mask(int64_t len, int64_t swa_valid_from, uint8_t* mask) {
+  for (int64_t p = 0; p < len; ++p) mask[p] = p >= swa_valid_from ? 1 : 0;
+  return ORC_OK;
+}
+
+/* Usable hit length on a cached prefix whose nodes carry dual indices (item 3): per token a Full Attention
+ * status and an SWA status.  A Full layer of the continuing request reads every position [0, L), so all of them
+ * need Full KV; an SWA layer reads the W - 1 positions before L, so those need SWA KV (item 1).  Evicting the
+ * SWA part of an old segment therefore costs nothing as long as the tail is intact, while a hole in the Full
+ * part ends the usable prefix there.  Returns the largest such L <= match_len. */
+int64_t orc_prefix_hit_len(int64_t match_len, int32_t window, const uint8_t* full_valid, const uint8_t* swa_valid) {
+  for (int64_t L = match_len; L > 0; --L) {
+    int ok = 1;
+    for (int64_t i = 0; i < L && ok; ++i)
+      if (!full_valid[i]) ok = 0;
+    int64_t lo = L - (window - 1);
+    if (lo < 0) lo = 0;
+    for (int64_t i = lo; i < L && ok; ++i)
+      if (!swa_valid[i]) ok = 0;
+    if (ok) return L;
+  }
+  return 0;
+}

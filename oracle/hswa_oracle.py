@@ -84,6 +84,10 @@ def _load():
         lib.orc_window_gather.restype = C.c_int
         lib.orc_window_scatter.restype = C.c_int
         lib.orc_attended_keys.restype = C.c_int64
+        lib.orc_swa_release.restype = C.c_int
+        lib.orc_release_due.restype = C.c_int
+        lib.orc_swa_valid_mask.restype = C.c_int
+        lib.orc_prefix_hit_len.restype = C.c_int64
         lib.orc_attended_keys.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
         _lib = lib
     return _lib
@@ -262,6 +266,41 @@ def window_scatter(cfg: OracleConfig, layer: OracleLayer, batch: OracleBatch, bu
     assert buf.shape == (batch.batch, cfg.window - 1, 2, cfg.num_kv_heads, cfg.head_dim)
     cc, cl, cb = cfg.c(), layer.c(), batch.c()
     _check(_load().orc_window_scatter(C.byref(cc), C.byref(cl), C.byref(cb), C.c_void_p(buf.ctypes.data)), "window_scatter")
+
+
+def swa_release(cfg: OracleConfig, ctx_len, release, swa_valid_from: np.ndarray):
+    """In-place update of int32 swa_valid_from after a step (ctx_len: lengths after the advance; release: uint8
+    flags per request or None for all)."""
+    assert swa_valid_from.dtype == np.int32
+    ctx = _i32(ctx_len)
+    rel = None if release is None else np.ascontiguousarray(release, dtype=np.uint8)
+    cc = cfg.c()
+    _check(_load().orc_swa_release(C.byref(cc), C.c_int32(ctx.shape[0]), C.c_void_p(ctx.ctypes.data),
+                                   None if rel is None else C.c_void_p(rel.ctypes.data),
+                                   C.c_void_p(swa_valid_from.ctypes.data)), "swa_release")
+
+
+RELEASE_CHUNK_END, RELEASE_REQUEST_END, RELEASE_DECODE_TOKEN = 0, 1, 2
+
+
+def release_due(kind: int, decoded: int = 0, every_n: int = 0) -> bool:
+    return bool(_load().orc_release_due(C.c_int32(kind), C.c_int64(decoded), C.c_int64(every_n)))
+
+
+def swa_valid_mask(length: int, swa_valid_from: int) -> np.ndarray:
+    mask = np.zeros(max(length, 1), dtype=np.uint8)
+    _check(_load().orc_swa_valid_mask(C.c_int64(length), C.c_int64(swa_valid_from), C.c_void_p(mask.ctypes.data)),
+           "swa_valid_mask")
+    return mask[:length]
+
+
+def prefix_hit_len(match_len: int, window: int, full_valid, swa_valid) -> int:
+    """Largest usable hit length <= match_len given per-token Full and SWA status of the cached prefix."""
+    f = np.ascontiguousarray(full_valid, dtype=np.uint8)
+    s = np.ascontiguousarray(swa_valid, dtype=np.uint8)
+    assert f.shape[0] >= match_len and s.shape[0] >= match_len
+    return int(_load().orc_prefix_hit_len(C.c_int64(match_len), C.c_int32(window), C.c_void_p(f.ctypes.data),
+                                          C.c_void_p(s.ctypes.data)))
 
 
 def num_threads() -> int:

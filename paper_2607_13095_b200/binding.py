@@ -27,6 +27,7 @@ EXPORTS = [
     "hswa_decode_attn", "hswa_decode_attn_mtp", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
     "hswa_window_safe_len", "hswa_swa_window_gather", "hswa_swa_window_scatter",
     "hswa_decode_workspace_need", "hswa_selftest_wait_timeout", "hswa_set_overlap",
+    "hswa_swa_release", "hswa_swa_valid_mask", "hswa_prefix_hit_len",
 ]
 
 
@@ -107,6 +108,12 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_swa_window_gather.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp]
     lib.hswa_swa_window_scatter.restype = C.c_int
     lib.hswa_swa_window_scatter.argtypes = [vp, C.POINTER(hswa_layer), C.POINTER(hswa_batch), vp, vp]
+    lib.hswa_swa_release.restype = C.c_int
+    lib.hswa_swa_release.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.hswa_swa_valid_mask.restype = C.c_int
+    lib.hswa_swa_valid_mask.argtypes = [vp, i32, vp, vp, i64, vp, vp]
+    lib.hswa_prefix_hit_len.restype = C.c_int64
+    lib.hswa_prefix_hit_len.argtypes = [i64, i32, vp, vp]
     lib.hswa_step_advance.restype = C.c_int
     lib.hswa_step_advance.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.hswa_get_async_error.restype = C.c_int
@@ -284,6 +291,29 @@ def hswa_swa_window_gather(h: Handle, layer: Layer, batch: Batch, buf: torch.Ten
 def hswa_swa_window_scatter(h: Handle, layer: Layer, batch: Batch, buf: torch.Tensor):
     _check(load().hswa_swa_window_scatter(h.ptr, C.byref(layer.c), C.byref(batch.c), _any_ptr(buf), _stream()),
            "hswa_swa_window_scatter")
+
+
+def hswa_swa_release(h: Handle, batch: int, ctx_len: torch.Tensor, release: Optional[torch.Tensor],
+                     swa_valid_from: torch.Tensor):
+    """release: uint8 CUDA tensor [B] (None: every request releases); swa_valid_from: int32 CUDA tensor [B], in place."""
+    assert swa_valid_from.dtype == torch.int32 and (release is None or release.dtype == torch.uint8)
+    _check(load().hswa_swa_release(h.ptr, batch, _ptr(ctx_len), _ptr(release), _ptr(swa_valid_from), _stream()),
+           "hswa_swa_release")
+
+
+def hswa_swa_valid_mask(h: Handle, batch: int, ctx_len: torch.Tensor, swa_valid_from: torch.Tensor, mask: torch.Tensor):
+    """mask: uint8 [B][stride], CUDA or pinned host."""
+    assert mask.dtype == torch.uint8 and mask.dim() == 2 and mask.shape[0] == batch
+    _check(load().hswa_swa_valid_mask(h.ptr, batch, _ptr(ctx_len), _ptr(swa_valid_from), int(mask.shape[1]), _any_ptr(mask),
+                                      _stream()), "hswa_swa_valid_mask")
+
+
+def hswa_prefix_hit_len(match_len: int, window: int, full_valid, swa_valid) -> int:
+    import numpy as np
+    f = np.ascontiguousarray(full_valid, dtype=np.uint8)
+    s = np.ascontiguousarray(swa_valid, dtype=np.uint8)
+    assert f.shape[0] >= match_len and s.shape[0] >= match_len
+    return int(load().hswa_prefix_hit_len(int(match_len), int(window), C.c_void_p(f.ctypes.data), C.c_void_p(s.ctypes.data)))
 
 
 def hswa_step_advance(h: Handle, batch: int, ctx_len: torch.Tensor, ring_head: torch.Tensor, q_indptr=None):

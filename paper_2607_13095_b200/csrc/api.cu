@@ -594,6 +594,37 @@ int64_t hswa_window_safe_len(int64_t match_len, int32_t window, const uint8_t* s
   return best;
 }
 
+int64_t hswa_prefix_hit_len(int64_t match_len, int32_t window, const uint8_t* full_valid, const uint8_t* swa_valid) {
+  if (match_len <= 0 || window < 1 || !full_valid) return 0;
+  // Full layers read every position below the hit length: the hit cannot pass the first token without Full KV
+  int64_t limit = 0;
+  while (limit < match_len && full_valid[limit]) ++limit;
+  if (window <= 1) return limit;
+  return hswa_window_safe_len(limit, window, swa_valid);
+}
+
+hswa_status hswa_swa_release(hswa_handle* h, int32_t batch, const int32_t* ctx_len, const uint8_t* release,
+                             int32_t* swa_valid_from, void* stream) {
+  if (h) h->chain_ok = 0;
+  if (!h || batch < 0) return HSWA_ERR_INVALID_ARG;
+  if (batch == 0) return HSWA_OK;
+  if (!ctx_len || !swa_valid_from) return HSWA_ERR_INVALID_ARG;
+  return hswa_launch_swa_release(model_params(h), batch, ctx_len, release, swa_valid_from, (cudaStream_t)stream) == cudaSuccess
+             ? HSWA_OK
+             : HSWA_ERR_CUDA;
+}
+
+hswa_status hswa_swa_valid_mask(hswa_handle* h, int32_t batch, const int32_t* ctx_len, const int32_t* swa_valid_from,
+                                int64_t mask_stride, uint8_t* mask, void* stream) {
+  if (h) h->chain_ok = 0;
+  if (!h || batch < 0 || mask_stride < 0) return HSWA_ERR_INVALID_ARG;
+  if (batch == 0 || mask_stride == 0) return HSWA_OK;
+  if (!ctx_len || !swa_valid_from || !mask) return HSWA_ERR_INVALID_ARG;
+  return hswa_launch_swa_valid_mask(batch, ctx_len, swa_valid_from, mask_stride, mask, (cudaStream_t)stream) == cudaSuccess
+             ? HSWA_OK
+             : HSWA_ERR_CUDA;
+}
+
 hswa_status hswa_step_advance(hswa_handle* h, int32_t batch, int32_t* ctx_len, int32_t* ring_head,
                               const int32_t* q_indptr, void* stream) {
   if (h) h->chain_ok = 0;

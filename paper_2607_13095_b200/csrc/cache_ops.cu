@@ -171,6 +171,47 @@ __global__ void __launch_bounds__(128) validate_kernel(ModelParams M, BatchParam
   }
 }
 
+// Out-of-window SWA release bookkeeping (paper Sec. 3.1.3 item 2).  swa_valid_from[r] is the first cached position
+// of request r whose SWA KV is still valid; the valid positions of a live request are the suffix
+// [swa_valid_from, ctx).  The ring overwrites everything older than C positions; a release (chunk end, request end,
+// every N decoded tokens: the caller's flags) drops everything the next token's window cannot reach.
+__global__ void swa_release_kernel(ModelParams M, int B, const int32_t* ctx_len, const uint8_t* release, int32_t* valid_from) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= B) return;
+  const int len = ctx_len[r];
+  int from = valid_from[r];
+  from = max(from, len - M.C);
+  if (release == nullptr || release[r]) from = max(from, len - (M.W - 1));
+  valid_from[r] = max(from, 0);
+}
+
+// Per-position SWA status: mask[r][p] = 1 iff swa_valid_from[r] <= p < ctx_len[r], 0 up to `stride`.  One thread
+// per 16 positions; blockIdx.y = request.  `mask` may be device memory or pinned host memory.
+__global__ void __launch_bounds__(256) swa_valid_mask_kernel(const int32_t* ctx_len, const int32_t* valid_from, int64_t stride,
+                                                             uint8_t* mask) {
+  const int r = blockIdx.y;
+  const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 16;
+  if (p0 >= stride) return;
+  const int64_t lo = valid_from[r], hi = ctx_len[r];
+  uint8_t* row = mask + (int64_t)r * stride;
+  if (p0 + 16 <= stride && ((reinterpret_cast<uintptr_t>(row + p0) & 15) == 0)) {
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t v = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int64_t p = p0 + j * 4 + b;
+        v |= (uint32_t)(p >= lo && p < hi) << (8 * b);
+      }
+      w[j] = v;
+    }
+    *reinterpret_cast<uint4*>(row + p0) = make_uint4(w[0], w[1], w[2], w[3]);
+  } else {
+    for (int64_t p = p0; p < min(p0 + 16, stride); ++p) row[p] = (p >= lo && p < hi) ? 1 : 0;
+  }
+}
+
 // Self-test of the bounded-wait path every pipeline kernel relies on: warp 1 waits, with the given limit, on an
 // mbarrier that warp 0 (the would-be producer) never arms.  The wait runs out, the waiter records
 // HSWA_ERR_TIMEOUT in the error word exactly as the pipeline kernels do, and the block returns normally:
@@ -216,6 +257,22 @@ cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int
                                  int32_t max_ctx_len, int32_t max_q_len, int32_t* err, cudaStream_t s) {
   if (b.B == 0) return cudaSuccess;
   validate_kernel<<<b.B, 128, 0, s>>>(m, b, is_swa, num_pages, max_ctx_len, max_q_len, err);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_swa_release(const ModelParams& m, int32_t B, const int32_t* ctx_len, const uint8_t* release,
+                                    int32_t* valid_from, cudaStream_t s) {
+  if (B == 0) return cudaSuccess;
+  swa_release_kernel<<<(B + 127) / 128, 128, 0, s>>>(m, B, ctx_len, release, valid_from);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_swa_valid_mask(int32_t B, const int32_t* ctx_len, const int32_t* valid_from, int64_t stride,
+                                       uint8_t* mask, cudaStream_t s) {
+  if (B == 0 || stride == 0) return cudaSuccess;
+  const int64_t threads = (stride + 15) / 16;
+  dim3 grid((unsigned)((threads + 255) / 256), B);
+  swa_valid_mask_kernel<<<grid, 256, 0, s>>>(ctx_len, valid_from, stride, mask);
   return cudaGetLastError();
 }
 

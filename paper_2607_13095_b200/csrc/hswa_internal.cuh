@@ -135,6 +135,10 @@ cudaError_t hswa_launch_window_move(const ModelParams& m, const BatchParams& b, 
                                     __nv_bfloat16* buf, int gather, int32_t* err, cudaStream_t s);
 cudaError_t hswa_launch_validate(const ModelParams& m, const BatchParams& b, int32_t is_swa, int64_t num_pages,
                                  int32_t max_ctx_len, int32_t max_q_len, int32_t* err, cudaStream_t s);
+cudaError_t hswa_launch_swa_release(const ModelParams& m, int32_t B, const int32_t* ctx_len, const uint8_t* release,
+                                    int32_t* valid_from, cudaStream_t s);
+cudaError_t hswa_launch_swa_valid_mask(int32_t B, const int32_t* ctx_len, const int32_t* valid_from, int64_t stride,
+                                       uint8_t* mask, cudaStream_t s);
 cudaError_t hswa_launch_wait_selftest(int64_t limit_clocks, int32_t* err, cudaStream_t s);
 
 #ifdef __CUDACC__

@@ -73,8 +73,10 @@ def test_mtp_rejects_rings_longer_than_three_tiles_without_launching():
         before = to_host_bits(swa.pool)
         q, k, v = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
         out = torch.full((t.batch, 2, d.num_q_heads, d.head_dim), 7.0, dtype=torch.float32, device="cuda")
+        b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None,
+                     max_q_len=1, total_q=t.batch, max_ctx_len=t.max_ctx_len)
         with pytest.raises(hb.HswaError) as e:
-            hb.hswa_decode_attn_mtp(h, swa, dev_batch(t, True), 2, q, k, v, out, None, workspace_for(h, t))
+            hb.hswa_decode_attn_mtp(h, swa, b, 2, q, k, v, out, None, workspace_for(h, t))
         assert e.value.status == hb.HSWA_ERR_UNSUPPORTED
         assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
         assert (out == 7.0).all() and np.array_equal(to_host_bits(swa.pool), before)   # nothing ran

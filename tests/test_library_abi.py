@@ -72,3 +72,20 @@ def test_window_safe_len_host():
             valid[: int(rng.integers(0, n))] = rng.integers(0, 2)
             m = int(rng.integers(0, n + 1))
             assert hb.hswa_window_safe_len(m, W, valid) == orc.window_safe_len(m, W, valid)
+
+
+def test_prefix_hit_len_is_host_arithmetic_and_matches_oracle():
+    import numpy as np
+    from oracle import hswa_oracle as orc
+    rng = np.random.default_rng(4)
+    for W in (1, 2, 4, 128):
+        for _ in range(80):
+            n = int(rng.integers(1, 400))
+            swa = (rng.random(n) < 0.9).astype(np.uint8)
+            swa[: int(rng.integers(0, n))] = 0
+            full = np.ones(n, np.uint8)
+            if rng.random() < 0.5:
+                full[int(rng.integers(0, n))] = 0
+            m = int(rng.integers(0, n + 1))
+            assert hb.hswa_prefix_hit_len(m, W, full, swa) == orc.prefix_hit_len(m, W, full, swa)
+    assert hb.load().hswa_prefix_hit_len(10, 4, None, None) == 0
