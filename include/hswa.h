@@ -189,8 +189,9 @@ hswa_status hswa_decode_attn_shared_prefix(hswa_handle* h, const hswa_layer* lay
  * and attends causally (to the cache and to new tokens 0..i; on SWA layers inside its own window).  The q_len
  * tokens end up appended (on a ring that requires q_len <= C - W + 1, checked: HSWA_ERR_INVALID_ARG): on Full
  * layers by an append launch ahead of one kernel that streams the KV once for all q_len tokens, on SWA layers
- * inside the attention kernel, which stages a ring once and gives every token its own warp (that needs the
- * whole ring in three 64-slot buffers: C > 192 with q_len > 1 is HSWA_ERR_UNSUPPORTED).  Workspace: as
+ * inside the attention kernel, which stages the ring (or, for rings of more than 192 slots, just the window) once
+ * for all tokens; a window of more than about 500 tokens on such a ring does not fit one block's shared memory:
+ * HSWA_ERR_UNSUPPORTED.  Workspace: as
  * hswa_decode_attn with max_total_q = max_batch * q_len.
  * After the step call hswa_step_advance with a q_indptr describing the ACCEPTED tokens per request. */
 hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const hswa_batch* batch, int32_t q_len,

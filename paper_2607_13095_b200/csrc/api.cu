@@ -410,8 +410,10 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   if (!q || !out || !k_new || !v_new) return HSWA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return HSWA_ERR_INVALID_ARG;
   if (layer->is_swa && q_len > h->ring_slots - h->cfg.window + 1) return HSWA_ERR_INVALID_ARG;  // append-then-attend limit
-  // the token mode of the ring kernel keeps a whole ring staged (three 64-slot buffers) while its warps patch and read it
-  if (layer->is_swa && (h->ring_slots + 63) / 64 > 3) return HSWA_ERR_UNSUPPORTED;
+  // The streaming ring kernel's token mode keeps a whole ring staged (three 64-slot buffers) while its warps patch and
+  // read it; longer rings take the compact-window kernel, which needs the window itself to fit shared memory
+  if (layer->is_swa && (h->ring_slots + 63) / 64 > 3 && !hswa_ring_compact_supported(model_params(h), q_len))
+    return HSWA_ERR_UNSUPPORTED;
   if (!layer->is_swa && (int64_t)b->max_ctx_len + q_len > (int64_t)b->max_blocks * h->cfg.page_size) return HSWA_ERR_INVALID_ARG;
 
   AppendParams a;

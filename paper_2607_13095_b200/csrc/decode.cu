@@ -1153,7 +1153,10 @@ cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool,
                                cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
   const int D = p.m.D, P = p.m.P;
-  if (p.is_swa) {  // rings: persistent blocks
+  if (p.is_swa) {
+    // persistent blocks streaming whole 64-slot ring tiles; a multi-token step needs the whole ring staged in the three
+    // stage buffers at once, so longer rings take the compact-window kernel
+    if (p.nq > 1 && (p.m.C + TK - 1) / TK > 3) return hswa_launch_decode_ring_compact(h, tm_pool, p, early_start, s);
     if (D == 128 && P == 64) return launch_ring_t<128, 64>(h, tm_pool, p, early_start, s);
     if (D == 128 && P == 32) return launch_ring_t<128, 32>(h, tm_pool, p, early_start, s);
     if (D == 128 && P == 16) return launch_ring_t<128, 16>(h, tm_pool, p, early_start, s);

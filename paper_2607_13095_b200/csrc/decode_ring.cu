@@ -1,0 +1,567 @@
+// SWA-layer decode over the ring of pages, compact-window form (paper Sec. 2.1: an SWA layer attends inside a window
+// of W keys; Sec. 3.1.1: strictly O(W) KV per request in a ring; Sec. 6.2: a decode step may carry draft tokens).
+//
+// This kernel serves multi-token decode steps on rings longer than the three 64-slot tiles the streaming ring kernel
+// (decode.cu) can keep staged at once; single-token steps and short rings stay on that kernel, which measured faster
+// (12 vs 15 us per layer at batch 64).
+//
+// Persistent blocks walk (request, KV head) items.  A block stages ONLY the 16-slot granules that meet the window in a
+// compact layout (72 KB of K and V at W = 128), three blocks per SM, and refills the K tiles of its next item as soon as
+// the scores of the current one exist, the V tiles as soon as its output accumulators are complete.
+//
+// Work split inside a block (4 warps, no producer / consumer roles):
+//   load      warp 0 works out the circular interval of visible slots [head - min(W - 1, ctx), head + nq - 1], one
+//             lane per granule issues the TMA tensor loads (128-byte swizzle), K and V on a barrier each;
+//   phase 1   split by keys: warp w computes S^T[keys x heads] = K Q^T (mma.sync m16n8k16, the GQA group's 8 heads
+//             are N = 8) for the 16-key blocks w, w + 4, ..., masks and scales them and publishes its partial row
+//             maxima; after a barrier (K is dead from here on) it turns its scores into P = 2^(S - m), rounds them to
+//             bf16 and leaves them in shared memory already in B-fragment order, with its partial row sums;
+//   phase 2   split by head dims: every warp accumulates O^T[its D / 4 dims x heads] += V^T P^T over ALL keys -- one
+//             8-byte load per 16 keys and token, one ldmatrix per MMA -- so no warp's result has to be merged with
+//             another's, and writes its rows straight from the accumulators.
+// Draft tokens (NT = 2 or 4 query tokens per request, causal among themselves) ride along as extra N columns: K and V
+// fragments are loaded once and multiplied with every token's Q / P.  The new tokens' K/V rows are patched into the
+// staged tiles and written to the cache here (fused append).  Rows of the staged tiles that hold slots outside every
+// token's window -- stale ring slots, possibly non-finite -- never count: their scores are masked and their V
+// fragments are zeroed after ldmatrix; a 16-key block wholly inside the window skips both.
+#include "hswa_internal.cuh"
+
+namespace {
+using namespace hswa_dev;
+
+constexpr int GR = HSWA_RING_GRANULE;  // slots per TMA box; divides every supported page size
+
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// The same m16n8k16 as mma_bf16_16816, as a pure function of its operands so that the compiler may interleave
+// independent accumulation chains.
+__device__ __forceinline__ void mma_pure(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D, int NT>
+__global__ void __launch_bounds__(128, NT == 1 ? 3 : 2)
+decode_ring_compact_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p, const int ng_max,
+                           const int k_region_bytes, const int n_items) {
+  constexpr int NW = 4;           // warps
+  constexpr int MT = D / 16 / NW; // 16-dim output blocks per warp
+  constexpr int HALVES = D / 64;
+  constexpr int KS = D / 16;      // k-steps of K Q^T
+  constexpr int CHUNKS = D / 8;   // 16-byte chunks per row
+  constexpr int NCOL = NT * 8;    // score columns: tokens x heads
+  constexpr int KB_REG = 3;       // 16-key blocks whose scores a warp can keep in registers
+  static_assert(2 * CHUNKS <= 32, "one chunk of a new K/V row per lane");
+
+  // All shared memory is one dynamic window (no static part, so that it starts on the 1 KB boundary the swizzled
+  // tiles need and three blocks fit an SM to the byte): K tiles | V tiles | P | scores (long windows) | small state.
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t smem_base = smem_u32(smem);
+
+  const ModelParams& M = p.m;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nq = p.nq;
+  const bool fuse = p.k_new != nullptr;
+  const int rows_max = ng_max * GR;
+  const int half_bytes = rows_max * 128;  // one 64-column half of K (or V)
+  const uint32_t aK = smem_base, aV = smem_base + k_region_bytes;
+  uint8_t* sK = smem;
+  uint8_t* sV = smem + k_region_bytes;
+  // Behind the V tiles: P (bf16, B-fragment order) [16-key block][NCOL][16], and for windows of more than
+  // KB_REG * NW granules, whose scores cannot wait in registers, a score area S [NCOL][sstr] fp32.
+  const bool s_in_regs = ng_max <= KB_REG * NW;
+  uint32_t* Pb = reinterpret_cast<uint32_t*>(smem + k_region_bytes + HALVES * half_bytes);
+  const int sstr = rows_max + 8;
+  float* S = reinterpret_cast<float*>(smem + k_region_bytes + HALVES * half_bytes + ng_max * NCOL * 32);
+  uint8_t* state = reinterpret_cast<uint8_t*>(S) + (s_in_regs ? 0 : NCOL * sstr * 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(state);                     // [2] K tiles landed, V tiles landed
+  float(*pm)[NCOL] = reinterpret_cast<float(*)[NCOL]>(state + 16);         // [NW] per-warp partial row maxima
+  float(*pl)[NCOL] = reinterpret_cast<float(*)[NCOL]>(state + 16 + NW * NCOL * 4);  // [NW] per-warp partial row sums
+  uint32_t* s_okm = reinterpret_cast<uint32_t*>(state + 16 + 2 * NW * NCOL * 4);    // [2] per item parity: granules loaded
+  int& s_abort = *reinterpret_cast<int*>(state + 16 + 2 * NW * NCOL * 4 + 8);       // a bounded wait ran out: all warps leave
+  const int ring_grans = M.C / GR;
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars[0]), 1);
+    mbar_init(smem_u32(&bars[1]), 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&tm_pool);
+    s_abort = 0;
+    if (smem_base & 1023u) {  // the swizzled tile addressing below assumes a 1 KB-aligned window
+      record_error(p.err, HSWA_ERR_CUDA, -1, (int)(smem_base & 1023u), 9);
+      s_abort = 1;
+    }
+  }
+  griddep_launch_dependents();  // the next kernel may begin its own cache loads (it waits before it touches q or out)
+  __syncthreads();
+  if (s_abort) return;
+
+  // ---- per-item state, fetched one item ahead ----
+  struct Meta {
+    int ctx, head, my_page;  // lane i keeps page id i of the ring
+  };
+  auto load_meta = [&](int item) {  // lengths, ring head and ring table are constant during a step
+    Meta m;
+    const int r = item / M.Hkv;
+    m.ctx = p.b.ctx_len[r];
+    m.head = p.b.ring_head[r];
+    m.my_page = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
+    return m;
+  };
+  // Warp 0: issue the TMA loads of one item's K (kv = 0) or V (kv = 1) tiles, one lane per granule.
+  auto issue_tiles = [&](int item, const Meta& m, int kv, int par) {
+    const int r = item / M.Hkv, kh = item % M.Hkv;
+    const int back = min(M.W - 1, m.ctx);
+    int start = m.head - back;
+    if (start < 0) start += M.C;
+    const int n_gran = min((start % GR + back + nq - 1) / GR + 1, ng_max);
+    int gi = start / GR + lane;
+    gi -= gi >= ring_grans ? ring_grans : 0;
+    gi -= gi >= ring_grans ? ring_grans : 0;  // lanes beyond the ring's granules do not load
+    const int slot_lo = gi * GR;
+    const int page = __shfl_sync(0xffffffffu, m.my_page, (slot_lo / M.P) & 31);
+    uint32_t okm = 0;
+    if (lane < n_gran) {
+      if (page < 0 || page >= p.num_pages) {
+        if (kv == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, slot_lo / M.P, page);
+      } else {
+        okm = 1u << lane;
+      }
+    }
+    okm = __reduce_or_sync(0xffffffffu, okm);
+    const uint32_t full_bar = smem_u32(&bars[kv]);
+    if (lane == 0) {
+      if (kv == 0) s_okm[par] = okm;
+      if (okm == 0)
+        mbar_arrive(full_bar);
+      else
+        mbar_arrive_expect_tx(full_bar, __popc(okm) * HALVES * GR * 128);
+    }
+    __syncwarp();
+    if ((okm >> lane) & 1u) {
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf)
+        tma_load_4d((kv == 0 ? aK : aV) + hf * half_bytes + lane * GR * 128, &tm_pool, full_bar, hf * 64, slot_lo % M.P,
+                    kv * M.Hkv + kh, page);
+    }
+  };
+  const int g_row = lane >> 2;  // head of this thread's B-fragment column
+  const int qd = (lane & 3) * 2;
+  const int mi = lane >> 3, mr = lane & 7;
+  uint32_t qf[NT][KS][2];
+  uint4 newrow[NT];
+  auto load_q = [&](int item) {
+    const int r = item / M.Hkv, kh = item % M.Hkv;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const bool live = nt < nq && g_row < M.G;
+      const __nv_bfloat16* qrow = p.q + (((int64_t)r * nq + (nt < nq ? nt : 0)) * M.Hq + kh * M.G + (g_row < M.G ? g_row : 0)) * D;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        qf[nt][ks][0] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+        qf[nt][ks][1] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+      }
+      if (fuse && lane < 2 * CHUNKS && nt < nq)
+        newrow[nt] = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) +
+                                                     (((int64_t)r * nq + nt) * M.Hkv + kh) * D + (lane % CHUNKS) * 8);
+    }
+  };
+
+  int it = blockIdx.x;
+  if (it >= n_items) return;
+  Meta mt_next = load_meta(it);
+  if (warp == 0) {
+    issue_tiles(it, mt_next, 0, 0);
+    issue_tiles(it, mt_next, 1, 0);
+  }
+  // q, k_new, v_new may be the previous kernel's output: nothing of them may be read before it has finished, but
+  // pulling their lines towards L2 (the point of coherence) early is harmless and takes DRAM latency off the chain
+  {
+    const int r = it / M.Hkv, kh = it % M.Hkv;
+    const char* qb = reinterpret_cast<const char*>(p.q + ((int64_t)r * nq * M.Hq + kh * M.G) * D);
+    if (threadIdx.x < M.G * D * 2 / 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(qb + threadIdx.x * 128));
+    if (fuse && threadIdx.x >= 64 && threadIdx.x < 64 + 2 * D * 2 / 128) {
+      const int j = threadIdx.x - 64, kv = j / (D * 2 / 128), o128 = j % (D * 2 / 128);
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>((kv == 0 ? p.k_new : p.v_new) +
+                                                                                    ((int64_t)r * nq * M.Hkv + kh) * D) + o128 * 128));
+    }
+  }
+  griddep_wait();
+  load_q(it);
+
+  for (int k = 0; it < n_items; ++k, it += gridDim.x) {
+    const int par = k & 1;
+    const int r = it / M.Hkv, kh = it % M.Hkv;
+    const Meta m = mt_next;
+    const int nxt = it + gridDim.x;
+    const bool has_next = nxt < n_items;
+    if (has_next) mt_next = load_meta(nxt);
+    const int ctx = m.ctx, head = m.head;
+    const int back = min(M.W - 1, ctx);  // cached positions token 0 can see
+    int start = head - back;             // ring slot of the oldest visible position
+    if (start < 0) start += M.C;
+    const int sr = start % GR;
+    const int last = back + nq - 1;      // offset of the newest token's slot from `start`
+    const int n_gran = min((sr + last) / GR + 1, ng_max);
+
+    bool ok = mbar_wait(smem_u32(&bars[0]), par);
+    if (!ok && lane == 0) {
+      record_error(p.err, HSWA_ERR_TIMEOUT, r, kh, 8);
+      *reinterpret_cast<volatile int*>(&s_abort) = 1;
+    }
+    const uint32_t okm = *reinterpret_cast<volatile uint32_t*>(&s_okm[par]);
+
+    // fused append: token nt sits at offset back + nt from `start`, i.e. in compact row sr + back + nt.  Every warp
+    // patches the rows (same bytes) so that it needs no block barrier before reading them; warp 0 writes the cache.
+    if (fuse && ok && lane < CHUNKS) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int row = sr + back + nt;
+        if (nt < nq && row < rows_max) *reinterpret_cast<uint4*>(sK + (lane >> 3) * half_bytes + swz128(row, lane & 7)) = newrow[nt];
+      }
+      fence_proxy_async_smem();  // a later TMA load overwrites these rows
+    }
+    __syncwarp();
+
+    // In compact rows: token nt sees [row_lo(nt), row_hi(nt)], any token sees [sr, sr + last]; rows of granules that
+    // were not loaded see nothing.
+    auto row_lo = [&](int nt) { return sr + max(0, back + nt - (M.W - 1)); };
+    auto row_hi = [&](int nt) { return sr + back + nt; };
+    auto visible = [&](int j, int nt) { return ((okm >> (j / GR)) & 1u) && j >= row_lo(nt) && j <= row_hi(nt); };
+    auto visible_any = [&](int j) { return ((okm >> (j / GR)) & 1u) && j >= sr && j <= sr + last; };
+    // is the 16-key block kb loaded and wholly inside [lo, hi]?  (same answer in every thread)
+    auto interior = [&](int kb, int lo, int hi) { return ((okm >> kb) & 1u) && kb * 16 >= lo && kb * 16 + 15 <= hi; };
+
+    // ---------------- phase 1a: scores of this warp's 16-key blocks, partial row maxima ----------------
+    float mx[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) mx[nt][0] = mx[nt][1] = -INFINITY;
+    auto score_block = [&](int kb, float (&sv)[NT][4]) {
+      // two accumulators per token halve the dependent MMA chain
+      float e[NT][4], f[NT][4];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) e[nt][c] = f[nt][c] = 0.f;
+      const int key = kb * 16 + (mi & 1) * 8 + mr;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int chunk = 2 * ks + (mi >> 1);
+        uint32_t a0, a1, a2, a3;
+        ldmatrix_x4(aK + (chunk >> 3) * half_bytes + swz128(key, chunk & 7), a0, a1, a2, a3);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) mma_pure((ks & 1) ? f[nt] : e[nt], a0, a1, a2, a3, qf[nt][ks][0], qf[nt][ks][1]);
+      }
+      const int keyA = kb * 16 + (lane >> 2), keyB = keyA + 8;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const bool inner = nt < nq && interior(kb, row_lo(nt), row_hi(nt));
+        const bool vA = inner || (nt < nq && visible(keyA, nt)), vB = inner || (nt < nq && visible(keyB, nt));
+        sv[nt][0] = vA ? (e[nt][0] + f[nt][0]) * M.scale_log2 : -INFINITY;
+        sv[nt][1] = vA ? (e[nt][1] + f[nt][1]) * M.scale_log2 : -INFINITY;
+        sv[nt][2] = vB ? (e[nt][2] + f[nt][2]) * M.scale_log2 : -INFINITY;
+        sv[nt][3] = vB ? (e[nt][3] + f[nt][3]) * M.scale_log2 : -INFINITY;
+        mx[nt][0] = fmaxf(mx[nt][0], fmaxf(sv[nt][0], sv[nt][2]));
+        mx[nt][1] = fmaxf(mx[nt][1], fmaxf(sv[nt][1], sv[nt][3]));
+      }
+    };
+    float s[KB_REG][NT][4];
+    if (s_in_regs) {
+#pragma unroll
+      for (int i = 0; i < KB_REG; ++i)
+        if (warp + NW * i < n_gran && ok) score_block(warp + NW * i, s[i]);
+    } else {
+      for (int kb = warp; kb < n_gran && ok; kb += NW) {
+        float sv[NT][4];
+        score_block(kb, sv);
+        const int keyA = kb * 16 + (lane >> 2);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float* row0 = S + (nt * 8 + qd) * sstr;
+          row0[keyA] = sv[nt][0];
+          row0[sstr + keyA] = sv[nt][1];
+          row0[keyA + 8] = sv[nt][2];
+          row0[sstr + keyA + 8] = sv[nt][3];
+        }
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        mx[nt][0] = fmaxf(mx[nt][0], __shfl_xor_sync(0xffffffffu, mx[nt][0], sh));
+        mx[nt][1] = fmaxf(mx[nt][1], __shfl_xor_sync(0xffffffffu, mx[nt][1], sh));
+      }
+      if (lane < 4) {
+        pm[warp][nt * 8 + qd] = mx[nt][0];
+        pm[warp][nt * 8 + qd + 1] = mx[nt][1];
+      }
+    }
+    // V rows of the new tokens, needed from phase 2 on (the V tiles may still be landing while phase 1 runs)
+    uint4 vrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) vrow[nt] = newrow[nt];
+    int new_page[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      int s_new = head + nt;
+      s_new -= s_new >= M.C ? M.C : 0;
+      new_page[nt] = __shfl_sync(0xffffffffu, m.my_page, (s_new / M.P) & 31);
+    }
+    // the cache copy of the new rows (warp 0: K from lanes [0, CHUNKS), V from lanes [CHUNKS, 2 CHUNKS))
+    if (fuse && ok && warp == 0 && lane < 2 * CHUNKS) {
+      const int kv = lane / CHUNKS, ch = lane % CHUNKS;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        if (nt >= nq) continue;
+        int s_new = head + nt;
+        s_new -= s_new >= M.C ? M.C : 0;
+        if (new_page[nt] < 0 || new_page[nt] >= p.num_pages) {
+          if (lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, new_page[nt]);
+        } else {
+          *reinterpret_cast<uint4*>(p.pool + ((((int64_t)new_page[nt] * 2 + kv) * M.Hkv + kh) * M.P + s_new % M.P) * D + ch * 8) =
+              newrow[nt];
+        }
+      }
+    }
+    // next item's Q and new rows: the registers are free from here on, the latency hides behind phases 1b and 2
+    if (has_next) load_q(nxt);
+    __syncthreads();  // every warp is done reading K and every partial maximum is published
+    if (*reinterpret_cast<volatile int*>(&s_abort)) return;
+    if (warp == 0 && has_next) issue_tiles(nxt, mt_next, 0, par ^ 1);  // the K tiles are dead: refill them
+
+    // ---------------- phase 1b: P = 2^(S - m) in bf16, B-fragment order, partial row sums ----------------
+    // This thread's accumulator columns are heads qd, qd + 1.  A B fragment of 16 keys x 8 columns wants, from the
+    // thread with (column g, t = lane mod 4), the word pairs {P[2t], P[2t+1]} and {P[2t+8], P[2t+9]} of column g: P is
+    // stored per (block, column) as 8 words in the order t0: {k0,k1},{k8,k9}; t1: {k2,k3},{k10,k11}; ... so phase 2
+    // reads 8 bytes per thread.  The accumulator holds keys kq = lane / 4 and kq + 8: neighbouring key lanes (kq even /
+    // odd) exchange values so that each writes one whole word.
+    float m_col[NT][2], lsum[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        float mm = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) mm = fmaxf(mm, pm[w][nt * 8 + qd + j]);
+        m_col[nt][j] = mm;
+        lsum[nt][j] = 0.f;
+      }
+    auto emit_block = [&](int kb, const float (&sv)[NT][4]) {
+      const int kq = lane >> 2;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float m0 = m_col[nt][0] == -INFINITY ? 0.f : m_col[nt][0], m1 = m_col[nt][1] == -INFINITY ? 0.f : m_col[nt][1];
+        // bf16 values the tensor core will multiply; sum exactly those
+        const uint32_t lo = pack_bf16x2(fast_exp2(sv[nt][0] - m0), fast_exp2(sv[nt][1] - m1));  // key kq: cols qd, qd + 1
+        const uint32_t hi = pack_bf16x2(fast_exp2(sv[nt][2] - m0), fast_exp2(sv[nt][3] - m1));  // key kq + 8
+        const float2 flo = unpack_bf16x2(lo), fhi = unpack_bf16x2(hi);
+        lsum[nt][0] += flo.x + fhi.x;
+        lsum[nt][1] += flo.y + fhi.y;
+        // partner lane holds key kq ^ 1, same columns
+        const uint32_t plo = __shfl_xor_sync(0xffffffffu, lo, 4), phi = __shfl_xor_sync(0xffffffffu, hi, 4);
+        // even kq writes column qd, odd kq writes column qd + 1: word {P[k even][col], P[k odd][col]}
+        const bool odd = kq & 1;
+        const uint32_t w_lo = odd ? __byte_perm(plo, lo, 0x7632) : __byte_perm(lo, plo, 0x5410);  // keys (kq & ~1, kq | 1)
+        const uint32_t w_hi = odd ? __byte_perm(phi, hi, 0x7632) : __byte_perm(hi, phi, 0x5410);  // keys + 8
+        const int col = nt * 8 + qd + (odd ? 1 : 0);
+        uint32_t* dst = Pb + ((size_t)(kb * NCOL + col)) * 8 + (kq >> 1) * 2;
+        *reinterpret_cast<uint2*>(dst) = make_uint2(w_lo, w_hi);
+      }
+    };
+    if (s_in_regs) {
+#pragma unroll
+      for (int i = 0; i < KB_REG; ++i)
+        if (warp + NW * i < n_gran && ok) emit_block(warp + NW * i, s[i]);
+    } else {
+      for (int kb = warp; kb < n_gran && ok; kb += NW) {
+        float sv[NT][4];
+        const int keyA = kb * 16 + (lane >> 2);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const float* row0 = S + (nt * 8 + qd) * sstr;
+          sv[nt][0] = row0[keyA];
+          sv[nt][1] = row0[sstr + keyA];
+          sv[nt][2] = row0[keyA + 8];
+          sv[nt][3] = row0[sstr + keyA + 8];
+        }
+        emit_block(kb, sv);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        lsum[nt][0] += __shfl_xor_sync(0xffffffffu, lsum[nt][0], sh);
+        lsum[nt][1] += __shfl_xor_sync(0xffffffffu, lsum[nt][1], sh);
+      }
+      if (lane < 4) {
+        pl[warp][nt * 8 + qd] = lsum[nt][0];
+        pl[warp][nt * 8 + qd + 1] = lsum[nt][1];
+      }
+    }
+    // the V tiles: wait, then patch in the new tokens' rows
+    if (ok && !mbar_wait(smem_u32(&bars[1]), par)) {
+      ok = false;
+      if (lane == 0) {
+        record_error(p.err, HSWA_ERR_TIMEOUT, r, kh, 9);
+        *reinterpret_cast<volatile int*>(&s_abort) = 1;
+      }
+    }
+    if (fuse && ok && lane >= CHUNKS && lane < 2 * CHUNKS) {
+      const int ch = lane - CHUNKS;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int row = sr + back + nt;
+        if (nt < nq && row < rows_max) *reinterpret_cast<uint4*>(sV + (ch >> 3) * half_bytes + swz128(row, ch & 7)) = vrow[nt];
+      }
+      fence_proxy_async_smem();
+    }
+    __syncthreads();  // P and the partial sums are complete
+    if (*reinterpret_cast<volatile int*>(&s_abort)) return;
+
+    // ---------------- phase 2: O^T[this warp's dims x heads] over all keys ----------------
+    float o[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) o[mt][nt][0] = o[mt][nt][1] = o[mt][nt][2] = o[mt][nt][3] = 0.f;
+    {
+      const uint32_t* pcol = Pb + (size_t)g_row * 8 + (lane & 3) * 2;
+      const int krow = (mi >> 1) * 8 + mr;
+      uint32_t v_addr[MT];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const int chunk = 2 * (warp * MT + mt) + (mi & 1);
+        v_addr[mt] = aV + (chunk >> 3) * half_bytes + swz128(krow, chunk & 7);  // + 2 KB per 16-key block
+      }
+#pragma unroll 3
+      for (int kb = 0; kb < n_gran; ++kb) {
+        uint2 b[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) b[nt] = *reinterpret_cast<const uint2*>(pcol + ((size_t)(kb * NCOL + nt * 8)) * 8);
+        // V^T fragments: a0 / a1 hold keys 16 kb + qd, qd + 1 in their halves, a2 / a3 keys 16 kb + 8 + qd, qd + 9.
+        // Rows no token can see may hold anything: zero them (0 x NaN would poison the sum); interior blocks have none.
+        uint32_t keep_lo = 0xffffffffu, keep_hi = 0xffffffffu;
+        if (!interior(kb, sr, sr + last)) {
+          const int k0 = kb * 16 + qd;
+          keep_lo = (visible_any(k0) ? 0x0000ffffu : 0u) | (visible_any(k0 + 1) ? 0xffff0000u : 0u);
+          keep_hi = (visible_any(k0 + 8) ? 0x0000ffffu : 0u) | (visible_any(k0 + 9) ? 0xffff0000u : 0u);
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(v_addr[mt] + kb * 2048, a0, a1, a2, a3);
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            mma_pure(o[mt][nt], a0 & keep_lo, a1 & keep_lo, a2 & keep_hi, a3 & keep_hi, b[nt].x, b[nt].y);
+        }
+      }
+    }
+    // row sums and maxima of this thread's accumulator columns (heads qd, qd + 1), read before the barrier below lets
+    // the next item overwrite them
+    float inv[NT][2], lse_v[NT][2];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        float l = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) l += pl[w][nt * 8 + qd + j];
+        inv[nt][j] = l > 0.f ? 1.f / l : 0.f;
+        lse_v[nt][j] = (p.lse && l > 0.f) ? (m_col[nt][j] + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      }
+    __syncthreads();  // every warp is done with the V tiles, P and the partial sums
+    if (warp == 0 && has_next) issue_tiles(nxt, mt_next, 1, par ^ 1);
+
+    // ---------------- output: straight from the accumulators ----------------
+    // (thread: heads qd, qd + 1; head dims 16 (warp MT + mt) + lane / 4 and + 8)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      if (nt >= nq) continue;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        if (qd + j >= M.G) continue;
+        const int64_t row = ((int64_t)r * nq + nt) * M.Hq + kh * M.G + qd + j;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int d0 = (warp * MT + mt) * 16 + (lane >> 2);
+          const float x = o[mt][nt][j] * inv[nt][j], y = o[mt][nt][2 + j] * inv[nt][j];
+          if (M.out_fp32) {
+            reinterpret_cast<float*>(p.out)[row * D + d0] = x;
+            reinterpret_cast<float*>(p.out)[row * D + d0 + 8] = y;
+          } else {
+            reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d0] = __float2bfloat16_rn(x);
+            reinterpret_cast<__nv_bfloat16*>(p.out)[row * D + d0 + 8] = __float2bfloat16_rn(y);
+          }
+        }
+        if (warp == 0 && (lane >> 2) == 0 && p.lse) p.lse[row] = lse_v[nt][j];
+      }
+    }
+  }
+}
+
+struct CompactPlan {
+  int ng_max, k_region, smem;
+};
+
+CompactPlan compact_plan(const ModelParams& m, int nq) {
+  const int D = m.D, NT = nq == 1 ? 1 : (nq == 2 ? 2 : 4);
+  CompactPlan c;
+  c.ng_max = (GR - 1 + m.W - 1 + nq - 1) / GR + 1;
+  const int rows_max = c.ng_max * GR;
+  const int tile = rows_max * D * 2;                                    // K (or V) tiles
+  const int p_area = c.ng_max * NT * 8 * 32;                              // P, bf16
+  const int s_area = c.ng_max <= 12 ? 0 : NT * 8 * (rows_max + 8) * 4;    // fp32 scores of long windows
+  c.k_region = (tile + 1023) & ~1023;
+  c.smem = c.k_region + tile + p_area + s_area + 16 + 2 * 4 * NT * 8 * 4 + 16;  // + barriers, partial maxima / sums, flags
+  return c;
+}
+
+template <int D, int NT>
+cudaError_t launch_compact_t(const CUtensorMap& tm, const DecodeParams& p, const CompactPlan& c, int sms, bool early_start,
+                             cudaStream_t s) {
+  auto kern = decode_ring_compact_kernel<D, NT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  const int n_items = p.b.B * p.m.Hkv;
+  const int resident = sms * (NT == 1 && c.smem <= 75 * 1024 ? 3 : (c.smem <= 112 * 1024 ? 2 : 1));
+  cfg.gridDim = dim3(n_items < resident ? n_items : resident, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = c.smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, tm, p, c.ng_max, c.k_region, n_items);
+}
+
+}  // namespace
+
+// Can the compact kernel serve this shape?  It needs the window's granules of one (request, KV head) in shared memory.
+bool hswa_ring_compact_supported(const ModelParams& m, int nq) {
+  if (m.P % GR != 0 || nq < 1 || nq > 4 || (m.D != 64 && m.D != 128)) return false;
+  const CompactPlan c = compact_plan(m, nq);
+  return c.ng_max <= 32 && c.smem <= 200 * 1024;
+}
+
+cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
+                                            bool early_start, cudaStream_t s) {
+  if (p.b.B == 0) return cudaSuccess;
+  const int D = p.m.D, nq = p.nq;
+  const int NT = nq == 1 ? 1 : (nq == 2 ? 2 : 4);
+  const CompactPlan c = compact_plan(p.m, nq);
+  if (D == 128 && NT == 1) return launch_compact_t<128, 1>(tm_pool, p, c, h->num_sms, early_start, s);
+  if (D == 128 && NT == 2) return launch_compact_t<128, 2>(tm_pool, p, c, h->num_sms, early_start, s);
+  if (D == 128 && NT == 4) return launch_compact_t<128, 4>(tm_pool, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 1) return launch_compact_t<64, 1>(tm_pool, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 2) return launch_compact_t<64, 2>(tm_pool, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 4) return launch_compact_t<64, 4>(tm_pool, p, c, h->num_sms, early_start, s);
+  return cudaErrorInvalidValue;
+}

@@ -115,6 +115,10 @@ cudaError_t hswa_launch_append(const AppendParams& p, cudaStream_t s);
 cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p, bool early_start,
                                cudaStream_t s);
 cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
+// SWA layers whose window fits shared memory: one block per (request, KV head) over a compact copy of the window
+bool hswa_ring_compact_supported(const ModelParams& m, int nq);
+cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
+                                            bool early_start, cudaStream_t s);
 cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
                                    bool early_start, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);

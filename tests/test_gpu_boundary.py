@@ -61,25 +61,63 @@ def test_exact_workspace_need_is_the_acceptance_threshold():
     assert np.abs(out.cpu().numpy() - ref).max() <= TOL
 
 
-def test_mtp_rejects_rings_longer_than_three_tiles_without_launching():
-    """Multi-token decode keeps a whole ring staged in three 64-slot buffers: a ring of more than 192 slots is
-    refused on the host (the single-token path serves it)."""
-    for d in (wl.Dims(num_q_heads=8, num_kv_heads=1, head_dim=128, page_size=64, window=200),   # R = 5, C = 320
-              wl.Dims(num_q_heads=8, num_kv_heads=1, head_dim=64, page_size=32, window=190)):   # R = 7, C = 224
-        sc = build_scenario(d, [500, 40], [2, 2], seed=42)
-        t = sc.tables
-        h = make_handle(d)
-        swa = hb.Layer(to_dev_bf16(sc.swa_pool), True)
-        before = to_host_bits(swa.pool)
-        q, k, v = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
-        out = torch.full((t.batch, 2, d.num_q_heads, d.head_dim), 7.0, dtype=torch.float32, device="cuda")
-        b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None,
-                     max_q_len=1, total_q=t.batch, max_ctx_len=t.max_ctx_len)
-        with pytest.raises(hb.HswaError) as e:
-            hb.hswa_decode_attn_mtp(h, swa, b, 2, q, k, v, out, None, workspace_for(h, t))
-        assert e.value.status == hb.HSWA_ERR_UNSUPPORTED
-        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
-        assert (out == 7.0).all() and np.array_equal(to_host_bits(swa.pool), before)   # nothing ran
+def test_mtp_rejects_windows_too_long_for_either_ring_kernel_without_launching():
+    """Multi-token decode on a ring needs the whole window staged at once.  Windows of a few hundred tokens fit the
+    compact kernel's shared memory; beyond that the streaming kernel only serves rings of at most three 64-slot
+    tiles, so such a shape is refused on the host (single-token decode still serves it)."""
+    d = wl.Dims(num_q_heads=8, num_kv_heads=1, head_dim=128, page_size=64, window=600)   # R = 11, C = 704
+    sc = build_scenario(d, [900, 40], [2, 2], seed=42)
+    t = sc.tables
+    h = make_handle(d)
+    swa = hb.Layer(to_dev_bf16(sc.swa_pool), True)
+    before = to_host_bits(swa.pool)
+    q, k, v = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    out = torch.full((t.batch, 2, d.num_q_heads, d.head_dim), 7.0, dtype=torch.float32, device="cuda")
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None,
+                 max_q_len=1, total_q=t.batch, max_ctx_len=t.max_ctx_len)
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn_mtp(h, swa, b, 2, q, k, v, out, None, workspace_for(h, t))
+    assert e.value.status == hb.HSWA_ERR_UNSUPPORTED
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert (out == 7.0).all() and np.array_equal(to_host_bits(swa.pool), before)   # nothing ran
+
+
+@pytest.mark.parametrize("W,P,D,G", [(200, 64, 128, 8), (190, 32, 64, 4), (33, 16, 128, 3), (64, 64, 64, 8), (1, 16, 64, 2),
+                                     (600, 64, 128, 8)])
+@pytest.mark.parametrize("nq", [1, 2, 3, 4])
+def test_ring_decode_other_windows_and_token_counts(W, P, D, G, nq):
+    """SWA decode for windows other than the paper's 128, every page size, one to four tokens per request, contexts
+    around every boundary (empty, shorter than the window, ring wrap)."""
+    d = wl.Dims(num_q_heads=G * 2, num_kv_heads=2, head_dim=D, page_size=P, window=W)
+    C = d.ring_slots
+    if nq > C - W + 1:
+        pytest.skip("append-then-attend limit of the ring")
+    if W == 600 and nq > 1:
+        pytest.skip("refused on the host: see the test above")
+    ctx = sorted({0, 1, 2, W - 2, W - 1, W, W + 1, P - 1, P, C - 1, C, C + 1, 3 * C + 5, 2000} - {-1})
+    B = len(ctx)
+    sc = build_scenario(d, ctx, [nq] * B, seed=48 + nq, ring_keep=C)
+    t = sc.tables
+    h = make_handle(d)
+    pool = to_dev_bf16(sc.swa_pool)
+    layer = hb.Layer(pool, True)
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None, max_q_len=1,
+                 total_q=B, max_ctx_len=t.max_ctx_len)
+    out = torch.full((B * nq, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((B * nq, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    q, k, v = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    if nq == 1:
+        hb.hswa_decode_attn(h, layer, b, q, k, v, out, lse, None)
+    else:
+        hb.hswa_decode_attn_mtp(h, layer, b, nq, q, k, v, out, lse, None)
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    ol = sc.layer(True)
+    ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
+    orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+    assert np.array_equal(to_host_bits(pool), ol.pool)
 
 
 def test_single_token_decode_serves_long_rings():
