@@ -544,14 +544,71 @@ def run_length_buckets(args, torch, device):
     bucketed = sorted(arrival, key=lambda i: reqs[i][0])  # stable: arrival order inside a tier
     t_mixed, t_bucket, t_bound = schedule(arrival), schedule(bucketed), float(ms.sum() / ranks)
     tokens = len(reqs) * chunk
+    balance = one_launch_balance(torch, device, reqs, arrival, bucketed, ranks)
     print(json.dumps({
         "metric": "prefill_attn_tokens_per_s_bucketed_vs_arrival_order", "unit": "x", "value": t_mixed / t_bucket,
         "chunk": chunk, "ranks": ranks, "requests": len(reqs), "n_gpus": 1, "data": "synthetic", "dtype": "bf16",
         "tokens_per_s": {"arrival_order": tokens / (t_mixed * 1e-3), "three_tier_buckets": tokens / (t_bucket * 1e-3),
                          "balanced_bound": tokens / (t_bound * 1e-3)},
         "block_ms_by_tier": [float(ms[[i for i, r_ in enumerate(reqs) if r_[0] == ti]].mean()) for ti in range(3)],
+        "one_launch_balance": balance,
         "note": "8 data-parallel attention ranks of one instance emulated one at a time on one GPU; a step costs its "
                 "slowest rank (per-layer synchronisation before the MoE stage); attention + append of one hybrid block"}))
+
+
+def one_launch_balance(torch, device, reqs, arrival, bucketed, per_batch, chunk=2048):
+    """The same requests batched 8 at a time into ONE Full-layer prefill launch each (a 2048-token chunk per request
+    over its cached prefix), in arrival order and bucketed by the paper's three tiers, with the blocks of a launch
+    handed out request by request and globally longest first.  Measured from per-block start / end stamps
+    (hswa_set_block_trace): the idle tail of an SM is the time between its last block's end and the launch's end;
+    reported as the mean over SMs, as a share of the launch's span, weighted by span over the launches."""
+    from paper_2607_13095_b200 import binding as hb
+    from paper_2607_13095_b200 import workloads as wl
+    d = wl.BIG
+    h = hb.Handle(d.num_q_heads, d.num_kv_heads, d.head_dim, d.page_size, d.window, d.ring_pages, 0.0, torch.bfloat16)
+    g = torch.Generator(device=device)
+    g.manual_seed(11)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+    res = {}
+    for sched_name, seq in (("arrival_order", arrival), ("three_tier_buckets", bucketed)):
+        acc = {m: {"span_ms": 0.0, "idle_ms": 0.0} for m in ("by_request", "longest_first")}
+        for i in range(0, len(seq), per_batch):
+            prefixes = [reqs[j][1] for j in seq[i:i + per_batch]]
+            t = wl.make_tables(d, prefixes, [chunk] * len(prefixes), seed=7, slack=1.0)
+            pool = torch.empty((t.num_full_pages, 2, d.num_kv_heads, d.page_size, d.head_dim), dtype=torch.bfloat16, device=device)
+            pool.normal_(generator=g)
+            layer = hb.Layer(pool, False)
+            T = t.total_q
+            q = torch.randn((T, d.num_q_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
+            k = torch.randn((T, d.num_kv_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
+            v = torch.randn((T, d.num_kv_heads, d.head_dim), generator=g, device=device, dtype=torch.bfloat16)
+            out = torch.empty((T, d.num_q_heads, d.head_dim), device=device, dtype=torch.bfloat16)
+            batch = hb.Batch(i32(t.ctx_len), i32(t.block_table), i32(t.ring_table), i32(t.ring_head), i32(t.q_indptr),
+                             max_q_len=t.max_q_len, total_q=T, max_ctx_len=t.max_ctx_len)
+            blocks = (d.group // 2) * d.num_kv_heads * t.batch * ((chunk + 127) // 128)
+            for mode_name, mode in (("by_request", hb.PREFILL_ORDER_BY_REQUEST), ("longest_first", hb.PREFILL_ORDER_LONGEST_FIRST)):
+                hb.hswa_set_prefill_order(h, mode)
+                trace = torch.zeros((blocks, 4), dtype=torch.int64, device=device)
+                hb.hswa_set_block_trace(h, trace)
+                hb.hswa_prefill_attn(h, layer, batch, q, k, v, False, out, None, None)
+                torch.cuda.synchronize()
+                hb.hswa_set_block_trace(h, None)
+                tr = trace.cpu().numpy()
+                tr = tr[tr[:, 1] > 0]
+                start, end = tr[:, 0].min(), tr[:, 1].max()
+                last_on_sm = np.array([tr[tr[:, 2] == s_, 1].max() for s_ in np.unique(tr[:, 2])])
+                acc[mode_name]["span_ms"] += float(end - start) * 1e-6
+                acc[mode_name]["idle_ms"] += float((end - last_on_sm).mean()) * 1e-6
+            del pool, q, k, v, out
+            torch.cuda.empty_cache()
+        res[sched_name] = {m: {"launch_ms_total": a_["span_ms"], "idle_tail_frac": a_["idle_ms"] / a_["span_ms"]}
+                           for m, a_ in acc.items()}
+    st = hb.hswa_get_async_error(h)
+    if st[0] != hb.HSWA_OK:
+        raise SystemExit(f"device error word set: {st}")
+    res["chunk"] = chunk
+    res["batch"] = per_batch
+    return res
 
 
 def run_layerwise_prefetch(args, torch, device):

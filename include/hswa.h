@@ -300,6 +300,23 @@ hswa_status hswa_get_async_error(hswa_handle* h, void* stream, int32_t info[4]);
 
 const char* hswa_status_string(hswa_status s);
 
+/* Work balance of mixed-length prefill batches (paper Sec. 5.3: requests whose cached prefixes differ a lot make
+ * the ranks / blocks that got the long ones finish last; the paper buckets by length, inside one launch the
+ * equivalent is the order in which blocks are handed out).
+ *
+ * hswa_set_prefill_order: order in which the Full-layer tile kernel of hswa_prefill_attn takes the (request,
+ * 128-token tile) pairs of a batch.  0: request by request, tiles ascending; 1: every request's last tile first,
+ * requests interleaved; 2 (default): globally longest first -- tile b of request r walks ceil(ctx[r] / 128) + b + 1
+ * key tiles, and the pairs are handed out in descending order of that count, computed on the device from ctx_len
+ * and q_indptr, so that the short ones fill the tail.  Results do not depend on the order.
+ *
+ * hswa_set_block_trace: debug aid.  With a device buffer int64 [capacity_blocks][4] set (NULL, 0 switches it off),
+ * every non-empty block of that kernel writes {start, end (nanoseconds of the GPU's global timer), SM id,
+ * request << 32 | tile} at its linear block index (x + gridDim.x * (y + gridDim.y * z)); blocks beyond the capacity write nothing.  The caller
+ * zeroes the buffer first and reads it after synchronising: the idle tail of every SM follows from it. */
+hswa_status hswa_set_prefill_order(hswa_handle* h, int32_t mode);
+hswa_status hswa_set_block_trace(hswa_handle* h, int64_t* buf, int64_t capacity_blocks);
+
 /* Self-test of the bounded waits (no paper counterpart; failure detection of the library itself).  Every wait
  * on a pipeline barrier inside the kernels gives up after a fixed number of SM clocks, records
  * HSWA_ERR_TIMEOUT in the error word and lets the block finish.  This call launches a one-block kernel whose

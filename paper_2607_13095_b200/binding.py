@@ -27,7 +27,7 @@ EXPORTS = [
     "hswa_decode_attn", "hswa_decode_attn_mtp", "hswa_decode_attn_shared_prefix", "hswa_decode_attn_static_ws", "hswa_prefill_attn", "hswa_step_advance", "hswa_get_async_error", "hswa_status_string",
     "hswa_window_safe_len", "hswa_swa_window_gather", "hswa_swa_window_scatter",
     "hswa_decode_workspace_need", "hswa_selftest_wait_timeout", "hswa_set_overlap",
-    "hswa_swa_release", "hswa_swa_valid_mask", "hswa_prefix_hit_len",
+    "hswa_swa_release", "hswa_swa_valid_mask", "hswa_prefix_hit_len", "hswa_set_prefill_order", "hswa_set_block_trace",
 ]
 
 
@@ -82,6 +82,10 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_workspace_bytes.argtypes = [vp, i32, i32, i32]
     lib.hswa_decode_workspace_need.restype = sz
     lib.hswa_decode_workspace_need.argtypes = [vp, i32, i32, i32, i32, i32]
+    lib.hswa_set_prefill_order.restype = C.c_int
+    lib.hswa_set_prefill_order.argtypes = [vp, i32]
+    lib.hswa_set_block_trace.restype = C.c_int
+    lib.hswa_set_block_trace.argtypes = [vp, vp, i64]
     lib.hswa_set_overlap.restype = C.c_int
     lib.hswa_set_overlap.argtypes = [vp, i32]
     lib.hswa_selftest_wait_timeout.restype = C.c_int
@@ -212,6 +216,22 @@ def hswa_decode_workspace_need(h: Handle, is_swa: bool, batch: int, max_ctx_len:
 
 def hswa_set_overlap(h: Handle, enabled: bool):
     _check(load().hswa_set_overlap(h.ptr, int(bool(enabled))), "hswa_set_overlap")
+
+
+PREFILL_ORDER_BY_REQUEST, PREFILL_ORDER_LAST_TILE_FIRST, PREFILL_ORDER_LONGEST_FIRST = 0, 1, 2
+
+
+def hswa_set_prefill_order(h: Handle, mode: int):
+    _check(load().hswa_set_prefill_order(h.ptr, int(mode)), "hswa_set_prefill_order")
+
+
+def hswa_set_block_trace(h: Handle, buf: Optional[torch.Tensor]):
+    """buf: int64 CUDA tensor [capacity][4] (zeroed by the caller) or None to switch the trace off."""
+    if buf is None:
+        _check(load().hswa_set_block_trace(h.ptr, None, 0), "hswa_set_block_trace")
+        return
+    assert buf.dtype == torch.int64 and buf.is_cuda and buf.is_contiguous() and buf.dim() == 2 and buf.shape[1] == 4
+    _check(load().hswa_set_block_trace(h.ptr, C.c_void_p(buf.data_ptr()), int(buf.shape[0])), "hswa_set_block_trace")
 
 
 def hswa_selftest_wait_timeout(h: Handle, limit_clocks: int):

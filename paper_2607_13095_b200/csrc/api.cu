@@ -202,6 +202,9 @@ hswa_status hswa_create(const hswa_config* cfg, hswa_handle** out) {
   h->chain_pool = nullptr;
   h->chain_ok = 0;
   h->overlap_enabled = 1;
+  h->prefill_order = 2;
+  h->trace = nullptr;
+  h->trace_cap = 0;
 
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -259,6 +262,19 @@ hswa_status hswa_set_overlap(hswa_handle* h, int32_t enabled) {
   if (!h) return HSWA_ERR_INVALID_ARG;
   h->overlap_enabled = enabled != 0;
   h->chain_ok = 0;
+  return HSWA_OK;
+}
+
+hswa_status hswa_set_prefill_order(hswa_handle* h, int32_t mode) {
+  if (!h || mode < 0 || mode > 2) return HSWA_ERR_INVALID_ARG;
+  h->prefill_order = mode;
+  return HSWA_OK;
+}
+
+hswa_status hswa_set_block_trace(hswa_handle* h, int64_t* buf, int64_t capacity_blocks) {
+  if (!h || capacity_blocks < 0 || (buf == nullptr) != (capacity_blocks == 0)) return HSWA_ERR_INVALID_ARG;
+  h->trace = reinterpret_cast<long long*>(buf);
+  h->trace_cap = capacity_blocks;
   return HSWA_OK;
 }
 
@@ -506,6 +522,9 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
   p.total_q = b->total_q;
   p.max_q_len = b->max_q_len;
   p.err = h->err;
+  p.order_mode = h->prefill_order;
+  p.trace = h->trace;
+  p.trace_cap = h->trace_cap;
   const int64_t tc_tiles = (int64_t)b->batch * ((b->max_q_len + 127) / 128);
   if (hswa_prefill_tc_supported(p.m) && b->q_indptr != nullptr && tc_tiles <= 65535) {
     // tcgen05 / TMEM / TMA tile kernel

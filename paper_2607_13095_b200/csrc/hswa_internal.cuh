@@ -29,6 +29,9 @@ struct hswa_handle {
   const void* chain_pool;  // pool of the previous fused decode: a kernel must not start early on the pool its predecessor writes
   int32_t chain_ok;
   int32_t overlap_enabled;  // hswa_set_overlap
+  int32_t prefill_order;    // hswa_set_prefill_order
+  long long* trace;         // hswa_set_block_trace: device int64 [trace_cap][4] or null
+  int64_t trace_cap;
 };
 
 // Model constants every kernel needs.
@@ -100,6 +103,9 @@ struct PrefillParams {
   int32_t total_q;
   int32_t max_q_len;
   int32_t* err;
+  int32_t order_mode;    // block order of the Full-layer tile kernel (hswa_set_prefill_order)
+  long long* trace;      // per-block {start ns, end ns, SM id, request << 32 | tile} (hswa_set_block_trace) or null
+  int64_t trace_cap;
   // shared-prefix stage of cascade decode only
   int32_t prefix_len;              // shared tokens (multiple of the page size)
   int32_t prefix_tiles_per_split;  // 128-key tiles per prefix slice

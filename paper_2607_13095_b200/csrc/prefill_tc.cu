@@ -174,6 +174,73 @@ __device__ __forceinline__ TileSeq tile_seq(int is_swa, int ctx, int b, int W, i
   return s;
 }
 
+// Global longest-first order of the (request, 128-token tile) pairs of a Full-layer prefill batch (paper Sec. 5.3:
+// mixed prefix lengths leave whoever got the long ones running last).  Tile b of request r walks
+// work(r, b) = ceil(ctx_r / 128) + b + 1 key tiles.  Pair number idx in descending order of work (ties: ascending
+// request) is found without sorting: count_ge(w), the number of pairs with work >= w, is a sum over requests of
+// clamped linear terms and falls with w, so a binary search finds the work value w* of pair idx, and idx minus
+// count_ge(w* + 1) says which of the requests that own a tile of exactly that work it is.  One warp, lanes strided
+// over requests; false when idx is beyond the last pair.
+__device__ __forceinline__ bool pick_longest_first(const BatchParams& bp, int idx, int lane, int* r_out, int* b_out) {
+  auto tiles_of = [&](int r, int& cr, int& nt) {
+    cr = (bp.ctx_len[r] + BN - 1) / BN;
+    nt = (bp.q_indptr[r + 1] - bp.q_indptr[r] + BM - 1) / BM;
+  };
+  auto count_ge = [&](int w) {
+    int c = 0;
+    for (int r = lane; r < bp.B; r += 32) {
+      int cr, nt;
+      tiles_of(r, cr, nt);
+      c += min(max(cr + nt - w + 1, 0), nt);
+    }
+#pragma unroll
+    for (int sh = 16; sh; sh >>= 1) c += __shfl_xor_sync(0xffffffffu, c, sh);
+    return c;
+  };
+  int w_max = 0;
+  for (int r = lane; r < bp.B; r += 32) {
+    int cr, nt;
+    tiles_of(r, cr, nt);
+    w_max = max(w_max, nt > 0 ? cr + nt : 0);
+  }
+#pragma unroll
+  for (int sh = 16; sh; sh >>= 1) w_max = max(w_max, __shfl_xor_sync(0xffffffffu, w_max, sh));
+  if (count_ge(1) <= idx) return false;
+  int lo = 1, hi = w_max + 1, above = 0;  // count_ge(lo) > idx >= count_ge(hi) = above
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    const int c = count_ge(mid);
+    if (c > idx) {
+      lo = mid;
+    } else {
+      hi = mid;
+      above = c;
+    }
+  }
+  int k = idx - above;  // rank among the pairs of work exactly lo
+  for (int base = 0; base < bp.B; base += 32) {
+    const int r = base + lane;
+    int cr = 0, nt = 0;
+    if (r < bp.B) tiles_of(r, cr, nt);
+    const unsigned has = __ballot_sync(0xffffffffu, r < bp.B && lo >= cr + 1 && lo <= cr + nt);
+    const int cnt = __popc(has);
+    if (k < cnt) {
+      const int sel = __fns(has, 0, k + 1);
+      *r_out = base + sel;
+      *b_out = lo - 1 - __shfl_sync(0xffffffffu, cr, sel);
+      return true;
+    }
+    k -= cnt;
+  }
+  return false;
+}
+
+__device__ __forceinline__ long long global_timer_ns() {
+  long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 // PREFIX = true turns the same pipeline into the shared-prefix stage of batched decode (paper Sec. 3.1.3 /
 // 3.1.4: requests that share a system prompt share its pages): the 128 rows of a Q tile are 16 requests x
 // the 8 query heads of one KV head, the keys are a slice of the shared prefix pages, nothing is masked, and
@@ -187,6 +254,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   __shared__ __align__(8) uint64_t bars[NUM_BARS];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int mma_abort;  // set by an MMA issuer that gave up, read by the other one
+  __shared__ int picked[2];  // (request, tile) of this block under the longest-first order; request -1: none
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
@@ -216,8 +284,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     ctx = p.prefix_len - tile_begin * BN;  // keys from this slice's first tile to the end of the prefix
     if (seq.nA <= 0) return;               // the host plans slices so that none is empty
   } else {
-    r = blockIdx.z % p.b.B;
-    b = max_tiles - 1 - (int)(blockIdx.z / p.b.B);  // longest tiles are scheduled first
+    if (p.order_mode == 2 && !p.is_swa) {
+      // globally longest first (on SWA layers every tile costs the same and the order does not matter)
+      if (warp == 0) {
+        int pr = -1, pb = 0;
+        if (!pick_longest_first(p.b, (int)blockIdx.z, lane, &pr, &pb)) pr = -1;
+        if (lane == 0) {
+          picked[0] = pr;
+          picked[1] = pb;
+        }
+      }
+      __syncthreads();
+      r = picked[0];
+      b = picked[1];
+      if (r < 0) return;  // uniform for the block
+    } else if (p.order_mode == 0) {
+      r = blockIdx.z / max_tiles;  // request by request, tiles ascending
+      b = blockIdx.z % max_tiles;
+    } else {
+      r = blockIdx.z % p.b.B;
+      b = max_tiles - 1 - (int)(blockIdx.z / p.b.B);  // every request's last (longest) tile first
+    }
     t0 = p.b.q_indptr[r];
     n = p.b.q_indptr[r + 1] - t0;
     if (b * BM >= n) return;  // uniform for the block
@@ -232,6 +319,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   __syncthreads();
   if (mma_abort) return;
   const int n_tiles = seq.total();
+  const int64_t trace_slot = blockIdx.x + (int64_t)gridDim.x * (blockIdx.y + (int64_t)gridDim.y * blockIdx.z);
+  const bool traced = p.trace != nullptr && trace_slot < p.trace_cap;
+  if (traced && threadIdx.x == 0) p.trace[trace_slot * 4] = global_timer_ns();
 
   auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
@@ -639,6 +729,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   if (warp == 8) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+  if (traced && threadIdx.x == 0) {
+    unsigned sm;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+    p.trace[trace_slot * 4 + 1] = global_timer_ns();
+    p.trace[trace_slot * 4 + 2] = sm;
+    p.trace[trace_slot * 4 + 3] = ((long long)r << 32) | (unsigned)b;
   }
 }
 

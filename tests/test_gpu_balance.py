@@ -1,0 +1,154 @@
+"""GPU tests of the mixed-length prefill work balance (paper Sec. 5.3) and of chunked prefill at the paper's longest
+prefixes (Sec. 5.2: a 16K chunk against up to 1M cached tokens): block order modes give identical results, the
+longest-first order is exactly the descending-work order, and the traced idle tail shrinks."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hswa_oracle as orc
+from paper_2607_13095_b200 import binding as hb
+from paper_2607_13095_b200 import workloads as wl
+from helpers import build_scenario, oracle_config
+from gpu_utils import dev_batch, dev_i32, make_handle, to_dev_bf16, to_host_bits
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def run_with_trace(h, layer, batch, q, k, v, out, blocks):
+    trace = torch.zeros((blocks, 4), dtype=torch.int64, device="cuda")
+    hb.hswa_set_block_trace(h, trace)
+    hb.hswa_prefill_attn(h, layer, batch, q, k, v, False, out, None, None)
+    torch.cuda.synchronize()
+    hb.hswa_set_block_trace(h, None)
+    t = trace.cpu().numpy()
+    return t[t[:, 1] > 0]   # non-empty blocks only
+
+
+def test_block_orders_agree_and_longest_first_is_descending_work():
+    d = wl.Dims(num_q_heads=16, num_kv_heads=2, head_dim=128, page_size=64)
+    ctx = [0, 4000, 130, 64, 9000, 127, 2500, 128, 0, 700, 33, 5000, 1, 129, 3000, 640, 0, 6000, 256, 255, 31, 900, 1500,
+           7000, 60, 61, 62, 63, 64, 65, 66, 67, 1000, 1001]                 # more than 32 requests: two ballot rounds
+    q_len = [300, 128, 129, 1, 127, 256, 64, 700, 0, 5, 130, 257, 400, 128, 0, 384, 512, 1, 2, 3, 640, 100, 200, 300,
+             128, 129, 130, 131, 132, 133, 134, 135, 136, 137]
+    sc = build_scenario(d, ctx, q_len, seed=95)
+    t = sc.tables
+    h = make_handle(d)
+    layer = hb.Layer(to_dev_bf16(sc.full_pool), False)
+    q, k, v = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    b = dev_batch(t, False)
+    max_tiles = (max(q_len) + 127) // 128
+    heads_x = d.group // 2
+    blocks = heads_x * d.num_kv_heads * t.batch * max_tiles
+    outs, traces = [], []
+    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LAST_TILE_FIRST, hb.PREFILL_ORDER_LONGEST_FIRST):
+        hb.hswa_set_prefill_order(h, mode)
+        out = torch.full((t.total_q, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+        traces.append(run_with_trace(h, layer, b, q, k, v, out, blocks))
+        outs.append(out.cpu().numpy())
+        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
+    assert np.abs(outs[0] - ref).max() <= TOL
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])   # the order changes no bit
+    # every (request, tile) pair ran exactly once per head pair and KV head, in every mode
+    pairs = sorted((r, bb) for r in range(t.batch) for bb in range((q_len[r] + 127) // 128))
+    for tr in traces:
+        got = sorted(zip((tr[:, 3] >> 32).tolist(), (tr[:, 3] & 0xffffffff).tolist()))
+        assert got == sorted(pairs * (heads_x * d.num_kv_heads))
+    # longest first: block z (the slow grid index) holds pair number z of the descending-work order, ties by request
+    work = lambda r, bb: (ctx[r] + 127) // 128 + bb + 1
+    want = sorted(pairs, key=lambda rb: (-work(*rb), rb[0]))
+    trace = torch.zeros((blocks, 4), dtype=torch.int64, device="cuda")
+    hb.hswa_set_prefill_order(h, hb.PREFILL_ORDER_LONGEST_FIRST)
+    hb.hswa_set_block_trace(h, trace)
+    out = torch.zeros((t.total_q, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+    hb.hswa_prefill_attn(h, layer, b, q, k, v, False, out, None, None)
+    torch.cuda.synchronize()
+    hb.hswa_set_block_trace(h, None)
+    tr = trace.cpu().numpy().reshape(t.batch * max_tiles, d.num_kv_heads, heads_x, 4)   # [z][y][x]
+    for z, (r, bb) in enumerate(want):
+        assert (tr[z, :, :, 3] >> 32 == r).all() and (tr[z, :, :, 3] & 0xffffffff == bb).all(), (z, r, bb)
+    assert (tr[len(want):, :, :, 1] == 0).all()   # grid slots beyond the last pair stay empty
+
+
+def test_longest_first_shrinks_the_idle_tail_of_a_mixed_length_batch():
+    """Eight requests whose cached prefixes span three orders of magnitude, one launch: with the long tiles handed out
+    last, most SMs sit idle while a few finish them; longest first leaves only short tiles for the tail."""
+    d = wl.BIG
+    ctx = [0, 1024, 4096, 16384, 32768, 65536, 131072, 262144]
+    chunk = 512
+    t = wl.make_tables(d, ctx, [chunk] * 8, seed=96, slack=1.0)
+    h = make_handle(d, out_dtype=torch.bfloat16)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(96)
+    pool = torch.empty((t.num_full_pages, 2, d.num_kv_heads, d.page_size, d.head_dim), dtype=torch.bfloat16, device="cuda")
+    pool.normal_(generator=g)
+    layer = hb.Layer(pool, False)
+    T = t.total_q
+    q = torch.randn((T, d.num_q_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    k = torch.randn((T, d.num_kv_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    v = torch.randn((T, d.num_kv_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    b = dev_batch(t, False)
+    blocks = (d.group // 2) * d.num_kv_heads * t.batch * (chunk // 128)
+    idle, outs = {}, {}
+    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LONGEST_FIRST):
+        hb.hswa_set_prefill_order(h, mode)
+        out = torch.zeros((T, d.num_q_heads, d.head_dim), dtype=torch.bfloat16, device="cuda")
+        run_with_trace(h, layer, b, q, k, v, out, blocks)          # warm-up
+        tr = run_with_trace(h, layer, b, q, k, v, out, blocks)
+        assert len(tr) == blocks
+        start, end = tr[:, 0].min(), tr[:, 1].max()
+        last_on_sm = np.array([tr[tr[:, 2] == s, 1].max() for s in np.unique(tr[:, 2])])
+        idle[mode] = float((end - last_on_sm).mean() / (end - start))   # mean idle tail of an SM, as a share of the span
+        outs[mode] = out.view(torch.int16).cpu().numpy()
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert np.array_equal(outs[hb.PREFILL_ORDER_BY_REQUEST], outs[hb.PREFILL_ORDER_LONGEST_FIRST])
+    assert idle[hb.PREFILL_ORDER_LONGEST_FIRST] < idle[hb.PREFILL_ORDER_BY_REQUEST], idle
+    assert idle[hb.PREFILL_ORDER_LONGEST_FIRST] < 0.10, idle
+
+
+@pytest.mark.parametrize("prefix", [262144, 1048576])
+def test_chunked_prefill_at_the_longest_prefixes(prefix):
+    """One request, a 16K-token chunk behind 256K / 1M cached tokens (paper Sec. 5.2's sweep): sampled rows of the Full
+    layer (first and last rows of the chunk, rows whose position sits on a page boundary, random others) and of the SWA
+    layer against the oracle; appended rows bit-exact.  Byte offsets pass 4 GB here."""
+    d = wl.BIG
+    chunk = 16384
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16e9:
+        pytest.skip("needs 16 GB of free device memory")
+    t = wl.make_tables(d, [prefix], [chunk], seed=97, slack=1.0)
+    assert t.num_full_pages * d.page_bytes > (1 << 32) or prefix < 1048576
+    h = make_handle(d, out_dtype=torch.bfloat16)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(97)
+    cfg = oracle_config(d)
+    ob = orc.OracleBatch(t.ctx_len, t.block_table, t.ring_table, t.ring_head, t.q_indptr)
+    q = torch.randn((chunk, d.num_q_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    k = torch.randn((chunk, d.num_kv_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    v = torch.randn((chunk, d.num_kv_heads, d.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    b = dev_batch(t, False)
+    rng = np.random.default_rng(97)
+    P = d.page_size
+    special = [0, 1, 127, 128, 129, (-prefix) % P, ((-prefix) % P) + P - 1, ((-prefix) % P) + P, chunk // 2, chunk - 2, chunk - 1]
+    for is_swa, n_rows in ((False, 256), (True, 512)):
+        n_pages = t.num_ring_pages if is_swa else t.num_full_pages
+        pool = torch.empty((n_pages, 2, d.num_kv_heads, P, d.head_dim), dtype=torch.bfloat16, device="cuda")
+        pool.normal_(generator=g)
+        before = to_host_bits(pool)
+        out = torch.zeros((chunk, d.num_q_heads, d.head_dim), dtype=torch.bfloat16, device="cuda")
+        hb.hswa_prefill_attn(h, hb.Layer(pool, is_swa), b, q, k, v, True, out, None, None)
+        torch.cuda.synchronize()
+        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+        tok = np.array(special + list(rng.integers(0, chunk, n_rows - len(special))), dtype=np.int32)
+        head = rng.integers(0, d.num_q_heads, len(tok)).astype(np.int32)
+        layer = orc.OracleLayer(before, is_swa)
+        ref, _ = orc.attention(cfg, layer, ob, to_host_bits(q), to_host_bits(k), to_host_bits(v), rows=(tok, head))
+        got = out.float().cpu().numpy()[tok, head]
+        err = np.abs(got - ref)
+        assert (err <= np.maximum(TOL, np.abs(ref) * 2.0 ** -8)).all(), (is_swa, float(err.max()))
+        orc.kv_append(cfg, layer, ob, to_host_bits(k), to_host_bits(v))
+        after = to_host_bits(pool)
+        assert np.array_equal(after, before), (is_swa, "pool bytes after the append")
+        del pool, before, after
+        torch.cuda.empty_cache()
