@@ -297,7 +297,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
       }
       __syncwarp();
     }
-    griddep_wait();  // this warp takes part in the output writes below
+    if (!p.late_dep_wait) griddep_wait();  // this warp takes part in the output writes below
   } else {
     // ---------------- consumers ----------------
     const int cw = warp - 1;
@@ -305,7 +305,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
     uint32_t qf[KS][2];
     // q, k_new, v_new may come from the previous kernel on the stream; the batch arrays and the cache that the
     // producer warp is already streaming do not
-    griddep_wait();
+    if (!p.late_dep_wait) griddep_wait();
     griddep_launch_dependents();
     {
       const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + g_row) * D;
@@ -421,6 +421,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
       if (d == 0) p.part_ml[row * p.max_splits + p.split_base + split] = make_float2(mm, L);
     }
   }
+  // Cascade decode: this grid must not be complete before the shared-prefix stage it overlapped is, because the
+  // combine waits for this grid only.
+  if (p.late_dep_wait) griddep_wait();
 }
 
 // Merge split-K partials: out = sum_s 2^(m_s - m) o_s / sum_s 2^(m_s - m) l_s.  One warp per (request, head).

@@ -70,6 +70,7 @@ struct DecodeParams {
   int32_t grid_splits; // splits this launch covers (grid extent)
   int32_t nq;          // new tokens per request (1; 2-4 for multi-token decode)
   int32_t max_ctx_len; // host-known bound of ctx_len the launch geometry was planned for
+  int32_t late_dep_wait;  // cascade decode: the dependency wait moves to the end of the block (see decode_kernel)
   float* part_o;       // [B*Hq][max_splits][D]
   float2* part_ml;     // [B*Hq][max_splits] (m in log2 units, l)
   int32_t* err;
