@@ -317,6 +317,13 @@ const char* hswa_status_string(hswa_status s);
 hswa_status hswa_set_prefill_order(hswa_handle* h, int32_t mode);
 hswa_status hswa_set_block_trace(hswa_handle* h, int64_t* buf, int64_t capacity_blocks);
 
+/* Read-bandwidth probe (no paper counterpart; a measuring aid).  Streams `bytes` of device memory at `buf`
+ * (128-byte aligned, a multiple of 32 KB) through shared memory with the same kind of bulk copies the decode
+ * kernels use and does nothing with them; timed by the caller with events, bytes / time is the practical ceiling
+ * for a read-only HBM stream on this GPU, which the roofline of paper Sec. 2.2's memory-bound decode is judged
+ * against next to the copy-based peak.  Asynchronous on `stream`. */
+hswa_status hswa_probe_read_stream(hswa_handle* h, const void* buf, size_t bytes, void* stream);
+
 /* Self-test of the bounded waits (no paper counterpart; failure detection of the library itself).  Every wait
  * on a pipeline barrier inside the kernels gives up after a fixed number of SM clocks, records
  * HSWA_ERR_TIMEOUT in the error word and lets the block finish.  This call launches a one-block kernel whose

@@ -28,6 +28,7 @@ EXPORTS = [
     "hswa_window_safe_len", "hswa_swa_window_gather", "hswa_swa_window_scatter",
     "hswa_decode_workspace_need", "hswa_selftest_wait_timeout", "hswa_set_overlap",
     "hswa_swa_release", "hswa_swa_valid_mask", "hswa_prefix_hit_len", "hswa_set_prefill_order", "hswa_set_block_trace",
+    "hswa_probe_read_stream",
 ]
 
 
@@ -86,6 +87,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.hswa_set_prefill_order.argtypes = [vp, i32]
     lib.hswa_set_block_trace.restype = C.c_int
     lib.hswa_set_block_trace.argtypes = [vp, vp, i64]
+    lib.hswa_probe_read_stream.restype = C.c_int
+    lib.hswa_probe_read_stream.argtypes = [vp, vp, sz, vp]
     lib.hswa_set_overlap.restype = C.c_int
     lib.hswa_set_overlap.argtypes = [vp, i32]
     lib.hswa_selftest_wait_timeout.restype = C.c_int
@@ -232,6 +235,11 @@ def hswa_set_block_trace(h: Handle, buf: Optional[torch.Tensor]):
         return
     assert buf.dtype == torch.int64 and buf.is_cuda and buf.is_contiguous() and buf.dim() == 2 and buf.shape[1] == 4
     _check(load().hswa_set_block_trace(h.ptr, C.c_void_p(buf.data_ptr()), int(buf.shape[0])), "hswa_set_block_trace")
+
+
+def hswa_probe_read_stream(h: Handle, buf: torch.Tensor):
+    """Stream a CUDA tensor's bytes (a multiple of 32 KB) through shared memory; time it with events."""
+    _check(load().hswa_probe_read_stream(h.ptr, _ptr(buf), buf.numel() * buf.element_size(), _stream()), "hswa_probe_read_stream")
 
 
 def hswa_selftest_wait_timeout(h: Handle, limit_clocks: int):

@@ -281,6 +281,12 @@ hswa_status hswa_set_block_trace(hswa_handle* h, int64_t* buf, int64_t capacity_
   return HSWA_OK;
 }
 
+hswa_status hswa_probe_read_stream(hswa_handle* h, const void* buf, size_t bytes, void* stream) {
+  if (!h || !buf || (reinterpret_cast<uintptr_t>(buf) & 127) != 0 || bytes % (32 * 1024) != 0) return HSWA_ERR_INVALID_ARG;
+  h->chain_ok = 0;
+  return hswa_launch_read_probe(buf, bytes, h->num_sms, h->err, (cudaStream_t)stream) == cudaSuccess ? HSWA_OK : HSWA_ERR_CUDA;
+}
+
 hswa_status hswa_selftest_wait_timeout(hswa_handle* h, int64_t limit_clocks, void* stream) {
   if (!h || limit_clocks < 1 || limit_clocks > 2000000000LL) return HSWA_ERR_INVALID_ARG;
   h->chain_ok = 0;

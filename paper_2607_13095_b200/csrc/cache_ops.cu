@@ -212,6 +212,41 @@ __global__ void __launch_bounds__(256) swa_valid_mask_kernel(const int32_t* ctx_
   }
 }
 
+// Read-bandwidth probe: the memory side of the Full-layer decode kernel without its arithmetic.  Persistent blocks
+// (two per SM, one warp each) stream their share of a buffer through a three-stage shared-memory ring with 32 KB bulk
+// copies completing on mbarriers; nobody looks at the bytes.  What this reaches is the practical ceiling for a kernel
+// that only reads HBM through TMA, which a copy-based peak (reads + writes) understates.
+constexpr int PROBE_CHUNK = 32 * 1024, PROBE_STAGES = 3;
+__global__ void __launch_bounds__(32) read_probe_kernel(const uint8_t* buf, long long chunks, int32_t* err) {
+  extern __shared__ __align__(128) uint8_t probe_smem[];
+  __shared__ __align__(8) uint64_t bars[PROBE_STAGES];
+  if (threadIdx.x != 0) return;
+  for (int i = 0; i < PROBE_STAGES; ++i) mbar_init(smem_u32(&bars[i]), 1);
+  mbar_fence_init();
+  long long k = 0;
+  for (long long c = blockIdx.x; c < chunks; c += gridDim.x, ++k) {
+    const int stage = (int)(k % PROBE_STAGES);
+    const uint32_t bar = smem_u32(&bars[stage]);
+    if (k >= PROBE_STAGES && !mbar_wait(bar, (uint32_t)((k / PROBE_STAGES - 1) & 1))) {  // the copy that used this stage
+      record_error(err, HSWA_ERR_TIMEOUT, -1, stage, 11);
+      return;
+    }
+    mbar_arrive_expect_tx(bar, PROBE_CHUNK);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(probe_smem + stage * PROBE_CHUNK)),
+                 "l"(buf + c * PROBE_CHUNK), "r"(PROBE_CHUNK), "r"(bar)
+                 : "memory");
+  }
+  // drain: no copy may be in flight when the block leaves
+  for (long long j = k > PROBE_STAGES ? k - PROBE_STAGES : 0; j < k; ++j) {
+    const int stage = (int)(j % PROBE_STAGES);
+    if (!mbar_wait(smem_u32(&bars[stage]), (uint32_t)((j / PROBE_STAGES) & 1))) {
+      record_error(err, HSWA_ERR_TIMEOUT, -1, stage, 12);
+      return;
+    }
+  }
+}
+
 // Self-test of the bounded-wait path every pipeline kernel relies on: warp 1 waits, with the given limit, on an
 // mbarrier that warp 0 (the would-be producer) never arms.  The wait runs out, the waiter records
 // HSWA_ERR_TIMEOUT in the error word exactly as the pipeline kernels do, and the block returns normally:
@@ -273,6 +308,17 @@ cudaError_t hswa_launch_swa_valid_mask(int32_t B, const int32_t* ctx_len, const 
   const int64_t threads = (stride + 15) / 16;
   dim3 grid((unsigned)((threads + 255) / 256), B);
   swa_valid_mask_kernel<<<grid, 256, 0, s>>>(ctx_len, valid_from, stride, mask);
+  return cudaGetLastError();
+}
+
+cudaError_t hswa_launch_read_probe(const void* buf, size_t bytes, int num_sms, int32_t* err, cudaStream_t s) {
+  const long long chunks = (long long)(bytes / PROBE_CHUNK);
+  if (chunks == 0) return cudaSuccess;
+  const int smem = PROBE_STAGES * PROBE_CHUNK;
+  cudaError_t e = cudaFuncSetAttribute(read_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  const long long want = 2LL * num_sms;
+  read_probe_kernel<<<(unsigned)(chunks < want ? chunks : want), 32, smem, s>>>(static_cast<const uint8_t*>(buf), chunks, err);
   return cudaGetLastError();
 }
 

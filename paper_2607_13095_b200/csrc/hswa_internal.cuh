@@ -150,6 +150,7 @@ cudaError_t hswa_launch_swa_release(const ModelParams& m, int32_t B, const int32
                                     int32_t* valid_from, cudaStream_t s);
 cudaError_t hswa_launch_swa_valid_mask(int32_t B, const int32_t* ctx_len, const int32_t* valid_from, int64_t stride,
                                        uint8_t* mask, cudaStream_t s);
+cudaError_t hswa_launch_read_probe(const void* buf, size_t bytes, int num_sms, int32_t* err, cudaStream_t s);
 cudaError_t hswa_launch_wait_selftest(int64_t limit_clocks, int32_t* err, cudaStream_t s);
 
 #ifdef __CUDACC__
