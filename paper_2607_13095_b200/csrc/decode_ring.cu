@@ -10,8 +10,12 @@
 // the scores of the current one exist, the V tiles as soon as its output accumulators are complete.
 //
 // Work split inside a block (4 warps, no producer / consumer roles):
-//   load      warp 0 works out the circular interval of visible slots [head - min(W - 1, ctx), head + nq - 1], one
-//             lane per granule issues the TMA tensor loads (128-byte swizzle), K and V on a barrier each;
+//   load      warp 0 works out the circular interval of visible slots [head - min(W - 1, ctx), head + nq - 1] and
+//             issues one TMA tensor load (128-byte swizzle) per run of granules that are consecutive inside a page --
+//             three runs for a window of 128 on pages of 64 -- with a tensor map per box height, K and V on a barrier
+//             each.  (Issuing a tensor load costs its thread on the order of a hundred cycles whatever the box size,
+//             and the copies of an SM are issued one after the other: 16-slot boxes, 36 per ring, made the issue
+//             itself the bottleneck.)
 //   phase 1   split by keys: warp w computes S^T[keys x heads] = K Q^T (mma.sync m16n8k16, the GQA group's 8 heads
 //             are N = 8) for the 16-key blocks w, w + 4, ..., masks and scales them and publishes its partial row
 //             maxima; after a barrier (K is dead from here on) it turns its scores into P = 2^(S - m), rounds them to
@@ -43,9 +47,14 @@ __device__ __forceinline__ void mma_pure(float (&c)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Tensor maps over one pool with boxes of 16, 32, 48 and 64 slots (only the heights up to a page are used).
+struct RingMaps {
+  CUtensorMap m[4];
+};
+
 template <int D, int NT>
 __global__ void __launch_bounds__(128, NT == 1 ? 3 : 2)
-decode_ring_compact_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p, const int ng_max,
+decode_ring_compact_kernel(const __grid_constant__ RingMaps maps, const DecodeParams p, const int ng_max,
                            const int k_region_bytes, const int n_items) {
   constexpr int NW = 4;           // warps
   constexpr int MT = D / 16 / NW; // 16-dim output blocks per warp
@@ -88,7 +97,7 @@ decode_ring_compact_kernel(const __grid_constant__ CUtensorMap tm_pool, const De
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
     mbar_fence_init();
-    tma_prefetch_desc(&tm_pool);
+    for (int i = 0; i < M.P / GR && i < 4; ++i) tma_prefetch_desc(&maps.m[i]);
     s_abort = 0;
     if (smem_base & 1023u) {  // the swizzled tile addressing below assumes a 1 KB-aligned window
       record_error(p.err, HSWA_ERR_CUDA, -1, (int)(smem_base & 1023u), 9);
@@ -122,13 +131,19 @@ decode_ring_compact_kernel(const __grid_constant__ CUtensorMap tm_pool, const De
     gi -= gi >= ring_grans ? ring_grans : 0;
     gi -= gi >= ring_grans ? ring_grans : 0;  // lanes beyond the ring's granules do not load
     const int slot_lo = gi * GR;
+    const int gpp = M.P / GR;  // granules per page
+    // a run: granules that follow each other inside one page; it starts at the interval's first granule and at every
+    // page boundary (the wrap to slot 0 is one)
+    const bool run_start = lane < n_gran && (lane == 0 || gi % gpp == 0);
+    const unsigned starts = __ballot_sync(0xffffffffu, run_start) | (1u << n_gran);
+    const int len = run_start ? __ffs(starts >> (lane + 1)) : 0;  // granules up to the next run
     const int page = __shfl_sync(0xffffffffu, m.my_page, (slot_lo / M.P) & 31);
     uint32_t okm = 0;
-    if (lane < n_gran) {
+    if (run_start) {
       if (page < 0 || page >= p.num_pages) {
         if (kv == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, slot_lo / M.P, page);
       } else {
-        okm = 1u << lane;
+        okm = ((1u << len) - 1u) << lane;
       }
     }
     okm = __reduce_or_sync(0xffffffffu, okm);
@@ -141,11 +156,11 @@ decode_ring_compact_kernel(const __grid_constant__ CUtensorMap tm_pool, const De
         mbar_arrive_expect_tx(full_bar, __popc(okm) * HALVES * GR * 128);
     }
     __syncwarp();
-    if ((okm >> lane) & 1u) {
+    if (run_start && ((okm >> lane) & 1u)) {
 #pragma unroll
       for (int hf = 0; hf < HALVES; ++hf)
-        tma_load_4d((kv == 0 ? aK : aV) + hf * half_bytes + lane * GR * 128, &tm_pool, full_bar, hf * 64, slot_lo % M.P,
-                    kv * M.Hkv + kh, page);
+        tma_load_4d((kv == 0 ? aK : aV) + hf * half_bytes + lane * GR * 128, &maps.m[len - 1], full_bar, hf * 64,
+                    slot_lo % M.P, kv * M.Hkv + kh, page);
     }
   };
   const int g_row = lane >> 2;  // head of this thread's B-fragment column
@@ -521,8 +536,25 @@ CompactPlan compact_plan(const ModelParams& m, int nq) {
   return c;
 }
 
+// 4-D views of the pool {D, P, 2 * Hkv, num_pages} with boxes {64, 16 k, 1, 1}, k = 1 .. P / 16, 128-byte swizzle.
+cudaError_t make_ring_maps(const hswa_handle* h, const DecodeParams& p, RingMaps* out) {
+  const ModelParams& m = p.m;
+  cuuint64_t dims[4] = {(cuuint64_t)m.D, (cuuint64_t)m.P, (cuuint64_t)(2 * m.Hkv), (cuuint64_t)p.num_pages};
+  cuuint64_t strides[3] = {(cuuint64_t)m.D * 2, (cuuint64_t)m.D * 2 * m.P, (cuuint64_t)m.D * 2 * m.P * 2 * m.Hkv};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 4; ++i) {
+    const int rows = (i + 1) * GR <= m.P ? (i + 1) * GR : GR;  // heights above a page are never used
+    cuuint32_t box[4] = {64, (cuuint32_t)rows, 1, 1};
+    if (h->encode_tiled(&out->m[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, p.pool, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  return cudaSuccess;
+}
+
 template <int D, int NT>
-cudaError_t launch_compact_t(const CUtensorMap& tm, const DecodeParams& p, const CompactPlan& c, int sms, bool early_start,
+cudaError_t launch_compact_t(const RingMaps& tm, const DecodeParams& p, const CompactPlan& c, int sms, bool early_start,
                              cudaStream_t s) {
   auto kern = decode_ring_compact_kernel<D, NT>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem);
@@ -548,7 +580,7 @@ cudaError_t launch_compact_t(const CUtensorMap& tm, const DecodeParams& p, const
 bool hswa_ring_compact_supported(const ModelParams& m, int nq) {
   if (m.P % GR != 0 || nq < 1 || nq > 4 || (m.D != 64 && m.D != 128)) return false;
   const CompactPlan c = compact_plan(m, nq);
-  return c.ng_max <= 32 && c.smem <= 200 * 1024;
+  return c.ng_max <= 31 && c.smem <= 200 * 1024;
 }
 
 cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
@@ -557,11 +589,15 @@ cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensor
   const int D = p.m.D, nq = p.nq;
   const int NT = nq == 1 ? 1 : (nq == 2 ? 2 : 4);
   const CompactPlan c = compact_plan(p.m, nq);
-  if (D == 128 && NT == 1) return launch_compact_t<128, 1>(tm_pool, p, c, h->num_sms, early_start, s);
-  if (D == 128 && NT == 2) return launch_compact_t<128, 2>(tm_pool, p, c, h->num_sms, early_start, s);
-  if (D == 128 && NT == 4) return launch_compact_t<128, 4>(tm_pool, p, c, h->num_sms, early_start, s);
-  if (D == 64 && NT == 1) return launch_compact_t<64, 1>(tm_pool, p, c, h->num_sms, early_start, s);
-  if (D == 64 && NT == 2) return launch_compact_t<64, 2>(tm_pool, p, c, h->num_sms, early_start, s);
-  if (D == 64 && NT == 4) return launch_compact_t<64, 4>(tm_pool, p, c, h->num_sms, early_start, s);
+  (void)tm_pool;  // the kernel uses its own maps, one per box height
+  RingMaps maps;
+  cudaError_t e = make_ring_maps(h, p, &maps);
+  if (e != cudaSuccess) return e;
+  if (D == 128 && NT == 1) return launch_compact_t<128, 1>(maps, p, c, h->num_sms, early_start, s);
+  if (D == 128 && NT == 2) return launch_compact_t<128, 2>(maps, p, c, h->num_sms, early_start, s);
+  if (D == 128 && NT == 4) return launch_compact_t<128, 4>(maps, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 1) return launch_compact_t<64, 1>(maps, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 2) return launch_compact_t<64, 2>(maps, p, c, h->num_sms, early_start, s);
+  if (D == 64 && NT == 4) return launch_compact_t<64, 4>(maps, p, c, h->num_sms, early_start, s);
   return cudaErrorInvalidValue;
 }
