@@ -559,7 +559,7 @@ def run_length_buckets(args, torch, device):
 def one_launch_balance(torch, device, reqs, arrival, bucketed, per_batch, chunk=2048):
     """The same requests batched 8 at a time into ONE Full-layer prefill launch each (a 2048-token chunk per request
     over its cached prefix), in arrival order and bucketed by the paper's three tiers, with the blocks of a launch
-    handed out request by request and globally longest first.  Measured from per-block start / end stamps
+    handed out request by request in batch order, longest request first (the default) and globally longest tile first.  Measured from per-block start / end stamps
     (hswa_set_block_trace): the idle tail of an SM is the time between its last block's end and the launch's end;
     reported as the mean over SMs, as a share of the launch's span, weighted by span over the launches."""
     from paper_2607_13095_b200 import binding as hb
@@ -571,7 +571,7 @@ def one_launch_balance(torch, device, reqs, arrival, bucketed, per_batch, chunk=
     i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
     res = {}
     for sched_name, seq in (("arrival_order", arrival), ("three_tier_buckets", bucketed)):
-        acc = {m: {"span_ms": 0.0, "idle_ms": 0.0} for m in ("by_request", "longest_first")}
+        acc = {m: {"span_ms": 0.0, "idle_ms": 0.0} for m in ("by_request", "longest_request_first", "longest_tile_first")}
         for i in range(0, len(seq), per_batch):
             prefixes = [reqs[j][1] for j in seq[i:i + per_batch]]
             t = wl.make_tables(d, prefixes, [chunk] * len(prefixes), seed=7, slack=1.0)
@@ -586,7 +586,9 @@ def one_launch_balance(torch, device, reqs, arrival, bucketed, per_batch, chunk=
             batch = hb.Batch(i32(t.ctx_len), i32(t.block_table), i32(t.ring_table), i32(t.ring_head), i32(t.q_indptr),
                              max_q_len=t.max_q_len, total_q=T, max_ctx_len=t.max_ctx_len)
             blocks = (d.group // 2) * d.num_kv_heads * t.batch * ((chunk + 127) // 128)
-            for mode_name, mode in (("by_request", hb.PREFILL_ORDER_BY_REQUEST), ("longest_first", hb.PREFILL_ORDER_LONGEST_FIRST)):
+            for mode_name, mode in (("by_request", hb.PREFILL_ORDER_BY_REQUEST),
+                                    ("longest_request_first", hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST),
+                                    ("longest_tile_first", hb.PREFILL_ORDER_LONGEST_TILE_FIRST)):
                 hb.hswa_set_prefill_order(h, mode)
                 trace = torch.zeros((blocks, 4), dtype=torch.int64, device=device)
                 hb.hswa_set_block_trace(h, trace)

@@ -305,10 +305,14 @@ const char* hswa_status_string(hswa_status s);
  * equivalent is the order in which blocks are handed out).
  *
  * hswa_set_prefill_order: order in which the Full-layer tile kernel of hswa_prefill_attn takes the (request,
- * 128-token tile) pairs of a batch.  0: request by request, tiles ascending; 1: every request's last tile first,
- * requests interleaved; 2 (default): globally longest first -- tile b of request r walks ceil(ctx[r] / 128) + b + 1
- * key tiles, and the pairs are handed out in descending order of that count, computed on the device from ctx_len
- * and q_indptr, so that the short ones fill the tail.  Results do not depend on the order.
+ * 128-token tile) pairs of a batch.  Tile b of request r walks ceil(ctx[r] / 128) + b + 1 key tiles.
+ *   0: request by request in batch order, tiles ascending;
+ *   1: every request's last tile first, requests interleaved;
+ *   2 (default): longest request first -- requests in descending order of their longest tile's work, the tiles of a
+ *      request together (their blocks share K/V pages in L2) and longest first, so that the launch ends on the
+ *      shortest tiles of the shortest request;
+ *   3: globally longest tile first, whatever its request.
+ * Orders 2 and 3 are computed on the device from ctx_len and q_indptr.  Results do not depend on the order.
  *
  * hswa_set_block_trace: debug aid.  With a device buffer int64 [capacity_blocks][4] set (NULL, 0 switches it off),
  * every non-empty block of that kernel writes {start, end (nanoseconds of the GPU's global timer), SM id,

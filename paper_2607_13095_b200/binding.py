@@ -221,7 +221,7 @@ def hswa_set_overlap(h: Handle, enabled: bool):
     _check(load().hswa_set_overlap(h.ptr, int(bool(enabled))), "hswa_set_overlap")
 
 
-PREFILL_ORDER_BY_REQUEST, PREFILL_ORDER_LAST_TILE_FIRST, PREFILL_ORDER_LONGEST_FIRST = 0, 1, 2
+PREFILL_ORDER_BY_REQUEST, PREFILL_ORDER_LAST_TILE_FIRST, PREFILL_ORDER_LONGEST_REQUEST_FIRST, PREFILL_ORDER_LONGEST_TILE_FIRST = 0, 1, 2, 3
 
 
 def hswa_set_prefill_order(h: Handle, mode: int):

@@ -269,7 +269,7 @@ hswa_status hswa_set_overlap(hswa_handle* h, int32_t enabled) {
 }
 
 hswa_status hswa_set_prefill_order(hswa_handle* h, int32_t mode) {
-  if (!h || mode < 0 || mode > 2) return HSWA_ERR_INVALID_ARG;
+  if (!h || mode < 0 || mode > 3) return HSWA_ERR_INVALID_ARG;
   h->prefill_order = mode;
   return HSWA_OK;
 }

@@ -235,6 +235,74 @@ __device__ __forceinline__ bool pick_longest_first(const BatchParams& bp, int id
   return false;
 }
 
+// Longest REQUEST first: the tiles of a request stay together (their blocks walk the same K/V pages at the same
+// time, which keeps them in L2 and measured 4 % faster on the chunked-prefill workload than any order that
+// interleaves requests), requests are taken in descending order of their longest tile's work, ceil(ctx_r / 128) +
+// tiles_r (ties: ascending request), and inside a request the longest tile goes first, so that the launch ends on the
+// shortest tiles of the shortest request.  Same search as above on T(w) = number of tiles of all requests whose key
+// is >= w.
+__device__ __forceinline__ bool pick_longest_request_first(const BatchParams& bp, int idx, int lane, int* r_out, int* b_out) {
+  auto tiles_of = [&](int r, int& key, int& nt) {
+    nt = (bp.q_indptr[r + 1] - bp.q_indptr[r] + BM - 1) / BM;
+    key = nt > 0 ? (bp.ctx_len[r] + BN - 1) / BN + nt : 0;
+  };
+  auto tiles_ge = [&](int w) {
+    int c = 0;
+    for (int r = lane; r < bp.B; r += 32) {
+      int key, nt;
+      tiles_of(r, key, nt);
+      c += key >= w ? nt : 0;
+    }
+#pragma unroll
+    for (int sh = 16; sh; sh >>= 1) c += __shfl_xor_sync(0xffffffffu, c, sh);
+    return c;
+  };
+  int w_max = 0;
+  for (int r = lane; r < bp.B; r += 32) {
+    int key, nt;
+    tiles_of(r, key, nt);
+    w_max = max(w_max, key);
+  }
+#pragma unroll
+  for (int sh = 16; sh; sh >>= 1) w_max = max(w_max, __shfl_xor_sync(0xffffffffu, w_max, sh));
+  if (tiles_ge(1) <= idx) return false;
+  int lo = 1, hi = w_max + 1, above = 0;  // tiles_ge(lo) > idx >= tiles_ge(hi) = above
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    const int c = tiles_ge(mid);
+    if (c > idx) {
+      lo = mid;
+    } else {
+      hi = mid;
+      above = c;
+    }
+  }
+  int k = idx - above;  // tile index among the requests whose key is exactly lo, taken in ascending request order
+  for (int base = 0; base < bp.B; base += 32) {
+    const int r = base + lane;
+    int key = 0, nt = 0;
+    if (r < bp.B) tiles_of(r, key, nt);
+    const int mine = key == lo ? nt : 0;
+    int incl = mine;  // inclusive prefix sum over the lanes
+#pragma unroll
+    for (int sh = 1; sh < 32; sh <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, sh);
+      if (lane >= sh) incl += v;
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (k < total) {
+      const unsigned hit = __ballot_sync(0xffffffffu, mine > 0 && k >= incl - mine && k < incl);
+      const int sel = __ffs(hit) - 1;
+      const int before = __shfl_sync(0xffffffffu, incl - mine, sel), ntile = __shfl_sync(0xffffffffu, nt, sel);
+      *r_out = base + sel;
+      *b_out = ntile - 1 - (k - before);  // longest tile first
+      return true;
+    }
+    k -= total;
+  }
+  return false;
+}
+
 __device__ __forceinline__ long long global_timer_ns() {
   long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -284,11 +352,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     ctx = p.prefix_len - tile_begin * BN;  // keys from this slice's first tile to the end of the prefix
     if (seq.nA <= 0) return;               // the host plans slices so that none is empty
   } else {
-    if (p.order_mode == 2 && !p.is_swa) {
-      // globally longest first (on SWA layers every tile costs the same and the order does not matter)
+    if (p.order_mode >= 2 && !p.is_swa) {
+      // longest request first (2) or globally longest tile first (3); on SWA layers every tile costs the same and the
+      // order does not matter
       if (warp == 0) {
         int pr = -1, pb = 0;
-        if (!pick_longest_first(p.b, (int)blockIdx.z, lane, &pr, &pb)) pr = -1;
+        const bool got = p.order_mode == 2 ? pick_longest_request_first(p.b, (int)blockIdx.z, lane, &pr, &pb)
+                                           : pick_longest_first(p.b, (int)blockIdx.z, lane, &pr, &pb);
+        if (!got) pr = -1;
         if (lane == 0) {
           picked[0] = pr;
           picked[1] = pb;

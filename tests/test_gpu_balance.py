@@ -1,6 +1,6 @@
 """GPU tests of the mixed-length prefill work balance (paper Sec. 5.3) and of chunked prefill at the paper's longest
 prefixes (Sec. 5.2: a 16K chunk against up to 1M cached tokens): block order modes give identical results, the
-longest-first order is exactly the descending-work order, and the traced idle tail shrinks."""
+device-computed orders are exactly the sorted orders they claim to be, and the traced idle tail shrinks."""
 import numpy as np
 import pytest
 import torch
@@ -41,7 +41,8 @@ def test_block_orders_agree_and_longest_first_is_descending_work():
     heads_x = d.group // 2
     blocks = heads_x * d.num_kv_heads * t.batch * max_tiles
     outs, traces = [], []
-    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LAST_TILE_FIRST, hb.PREFILL_ORDER_LONGEST_FIRST):
+    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LAST_TILE_FIRST, hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST,
+                 hb.PREFILL_ORDER_LONGEST_TILE_FIRST):
         hb.hswa_set_prefill_order(h, mode)
         out = torch.full((t.total_q, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
         traces.append(run_with_trace(h, layer, b, q, k, v, out, blocks))
@@ -49,31 +50,35 @@ def test_block_orders_agree_and_longest_first_is_descending_work():
         assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
     ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
     assert np.abs(outs[0] - ref).max() <= TOL
-    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])   # the order changes no bit
+    assert all(np.array_equal(outs[0], o) for o in outs[1:])   # the order changes no bit
     # every (request, tile) pair ran exactly once per head pair and KV head, in every mode
     pairs = sorted((r, bb) for r in range(t.batch) for bb in range((q_len[r] + 127) // 128))
     for tr in traces:
         got = sorted(zip((tr[:, 3] >> 32).tolist(), (tr[:, 3] & 0xffffffff).tolist()))
         assert got == sorted(pairs * (heads_x * d.num_kv_heads))
-    # longest first: block z (the slow grid index) holds pair number z of the descending-work order, ties by request
+    # the two device-computed orders, pair by pair: block z (the slow grid index) holds pair number z
     work = lambda r, bb: (ctx[r] + 127) // 128 + bb + 1
-    want = sorted(pairs, key=lambda rb: (-work(*rb), rb[0]))
-    trace = torch.zeros((blocks, 4), dtype=torch.int64, device="cuda")
-    hb.hswa_set_prefill_order(h, hb.PREFILL_ORDER_LONGEST_FIRST)
-    hb.hswa_set_block_trace(h, trace)
-    out = torch.zeros((t.total_q, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
-    hb.hswa_prefill_attn(h, layer, b, q, k, v, False, out, None, None)
-    torch.cuda.synchronize()
-    hb.hswa_set_block_trace(h, None)
-    tr = trace.cpu().numpy().reshape(t.batch * max_tiles, d.num_kv_heads, heads_x, 4)   # [z][y][x]
-    for z, (r, bb) in enumerate(want):
-        assert (tr[z, :, :, 3] >> 32 == r).all() and (tr[z, :, :, 3] & 0xffffffff == bb).all(), (z, r, bb)
-    assert (tr[len(want):, :, :, 1] == 0).all()   # grid slots beyond the last pair stay empty
+    tiles = lambda r: (q_len[r] + 127) // 128
+    by_tile = sorted(pairs, key=lambda rb: (-work(*rb), rb[0]))                                   # longest tile first
+    by_request = sorted(pairs, key=lambda rb: (-work(rb[0], tiles(rb[0]) - 1), rb[0], -rb[1]))    # longest request first
+    for mode, want in ((hb.PREFILL_ORDER_LONGEST_TILE_FIRST, by_tile), (hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST, by_request)):
+        trace = torch.zeros((blocks, 4), dtype=torch.int64, device="cuda")
+        hb.hswa_set_prefill_order(h, mode)
+        hb.hswa_set_block_trace(h, trace)
+        out = torch.zeros((t.total_q, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
+        hb.hswa_prefill_attn(h, layer, b, q, k, v, False, out, None, None)
+        torch.cuda.synchronize()
+        hb.hswa_set_block_trace(h, None)
+        tr = trace.cpu().numpy().reshape(t.batch * max_tiles, d.num_kv_heads, heads_x, 4)   # [z][y][x]
+        for z, (r, bb) in enumerate(want):
+            assert (tr[z, :, :, 3] >> 32 == r).all() and (tr[z, :, :, 3] & 0xffffffff == bb).all(), (mode, z, r, bb)
+        assert (tr[len(want):, :, :, 1] == 0).all()   # grid slots beyond the last pair stay empty
 
 
 def test_longest_first_shrinks_the_idle_tail_of_a_mixed_length_batch():
     """Eight requests whose cached prefixes span three orders of magnitude, one launch: with the long tiles handed out
-    last, most SMs sit idle while a few finish them; longest first leaves only short tiles for the tail."""
+    last, most SMs sit idle while a few finish them; with the longest request (or tile) first only short tiles are left
+    for the tail."""
     d = wl.BIG
     ctx = [0, 1024, 4096, 16384, 32768, 65536, 131072, 262144]
     chunk = 512
@@ -91,7 +96,7 @@ def test_longest_first_shrinks_the_idle_tail_of_a_mixed_length_batch():
     b = dev_batch(t, False)
     blocks = (d.group // 2) * d.num_kv_heads * t.batch * (chunk // 128)
     idle, outs = {}, {}
-    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LONGEST_FIRST):
+    for mode in (hb.PREFILL_ORDER_BY_REQUEST, hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST, hb.PREFILL_ORDER_LONGEST_TILE_FIRST):
         hb.hswa_set_prefill_order(h, mode)
         out = torch.zeros((T, d.num_q_heads, d.head_dim), dtype=torch.bfloat16, device="cuda")
         run_with_trace(h, layer, b, q, k, v, out, blocks)          # warm-up
@@ -102,9 +107,10 @@ def test_longest_first_shrinks_the_idle_tail_of_a_mixed_length_batch():
         idle[mode] = float((end - last_on_sm).mean() / (end - start))   # mean idle tail of an SM, as a share of the span
         outs[mode] = out.view(torch.int16).cpu().numpy()
     assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
-    assert np.array_equal(outs[hb.PREFILL_ORDER_BY_REQUEST], outs[hb.PREFILL_ORDER_LONGEST_FIRST])
-    assert idle[hb.PREFILL_ORDER_LONGEST_FIRST] < idle[hb.PREFILL_ORDER_BY_REQUEST], idle
-    assert idle[hb.PREFILL_ORDER_LONGEST_FIRST] < 0.10, idle
+    for mode in (hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST, hb.PREFILL_ORDER_LONGEST_TILE_FIRST):
+        assert np.array_equal(outs[hb.PREFILL_ORDER_BY_REQUEST], outs[mode])
+        assert idle[mode] < idle[hb.PREFILL_ORDER_BY_REQUEST], idle
+        assert idle[mode] < 0.10, idle
 
 
 @pytest.mark.parametrize("prefix", [262144, 1048576])
