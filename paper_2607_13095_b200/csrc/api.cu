@@ -560,11 +560,13 @@ hswa_status hswa_prefill_attn(hswa_handle* h, const hswa_layer* layer, const hsw
       CUtensorMap pq, pk, pv;
       if ((st = make_rows_map(h, q, h->cfg.num_q_heads, b->total_q, tq, &pq, h->group)) != HSWA_OK) return st;
       if (h->group == 8 && h->cfg.window == 128) {
-        // pipelined kernel (its mask shortcuts assume the paper's W = 128): 128-token blocks, K/V through the 128-row boxes of the tile kernel's maps
-        CUtensorMap po = pq;
+        // streaming kernel (its mask shortcuts assume the paper's W = 128): K/V arrive in 16-row pieces
+        CUtensorMap po = pq, k16, v16;
         const int tma_out = h->cfg.out_dtype == 0;  // bf16 output leaves through a TMA tensor store
         if (tma_out && (st = make_rows_map(h, out, h->cfg.num_q_heads, b->total_q, tq, &po, h->group)) != HSWA_OK) return st;
-        if (hswa_launch_prefill_swa_pipe(pq, tm_k, tm_v, po, tma_out, p, split_tiles, (cudaStream_t)stream) != cudaSuccess)
+        if ((st = make_rows_map(h, k_new, h->cfg.num_kv_heads, b->total_q, 16, &k16)) != HSWA_OK) return st;
+        if ((st = make_rows_map(h, v_new, h->cfg.num_kv_heads, b->total_q, 16, &v16)) != HSWA_OK) return st;
+        if (hswa_launch_prefill_swa_stream(pq, k16, v16, po, tma_out, p, h->num_sms, (cudaStream_t)stream) != cudaSuccess)
           return HSWA_ERR_CUDA;
       } else {
         if ((st = make_rows_map(h, k_new, h->cfg.num_kv_heads, b->total_q, nkeys, &pk)) != HSWA_OK) return st;

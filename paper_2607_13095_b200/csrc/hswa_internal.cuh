@@ -135,9 +135,9 @@ cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap
 void hswa_prefill_packed_geometry(int G, int* tq, int* nkeys);
 cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const PrefillParams& p, int n_slices,
                                       cudaStream_t s);
-cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                         const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int first_block,
-                                         cudaStream_t s);
+cudaError_t hswa_launch_prefill_swa_stream(const CUtensorMap& tm_q, const CUtensorMap& tm_k16, const CUtensorMap& tm_v16,
+                                           const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int num_sms,
+                                           cudaStream_t s);
 cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                            const PrefillParams& p, int first_tok, cudaStream_t s);
 cudaError_t hswa_launch_advance(const ModelParams& m, int32_t B, int32_t* ctx_len, int32_t* ring_head,
@@ -183,6 +183,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       "{\n"
       ".reg .pred p;\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Non-blocking test of a phase.  try_wait above may suspend the thread for a hardware-chosen time when the phase
+// has not completed, which is right for a thread with one thing to wait for; a thread that polls several barriers
+// in turn (whichever is ready first) must use this one, or it sleeps on one barrier while another completes.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)

@@ -1016,60 +1016,122 @@ cudaError_t launch_packed(const CUtensorMap& tm_q, const CUtensorMap& tm_k, cons
 
 
 // ---------------------------------------------------------------------------------------------------------
-// SWA layers, GQA group of 8, tokens whose whole window lies inside the chunk: pipelined variant of the packed
-// kernel.  One block = 128 consecutive tokens of one (request, KV head).  The 256 chunk keys those tokens can
-// see are loaded once (K and V, 64 KB each); the block then walks eight sub-tiles of 16 tokens x 8 heads
-// (128 rows) against a 144-key slice of that buffer that slides by 16 rows per sub-tile.  Two softmax
-// warpgroups alternate sub-tiles, each with its own Q buffer and its own 256 TMEM columns (S in [0, 144), P
-// over its first 72 columns, O in [128, 256)), so the Q load, the S MMA, the softmax, the PV MMA and the
-// output of neighbouring sub-tiles overlap and K/V traffic is paid once per 128 tokens.
-namespace pipe {
+// SWA layers, GQA group of 8, window 128, tokens whose whole window lies inside the chunk: streaming kernel.
+// Persistent blocks walk long runs of 16-token sub-tiles of one (request, KV head) stream.  A sub-tile is 16
+// tokens x 8 heads (128 rows) against the 144 keys its tokens can see (16 + 127, rounded up to 16).  K and V live
+// in a CIRCULAR buffer of 256 key rows (16 slots of 16): sub-tile s (tokens [i, i + 16), i = 128 + 16 s) needs
+// keys [i - 128, i + 16), of which only [i, i + 16) are new, so every sub-tile loads its Q tile (32 KB), ONE
+// 16-key piece of K and of V (4 KB each) into the slot of the keys that fell out of every window eight sub-tiles
+// ago, and stores 32 KB: each key is read once per stream.  The 144-key slice starts at row (i - 128) mod 256 and
+// may wrap: the S MMA is then issued as two groups (N1 + N2 keys, adjacent TMEM columns), and the PV k-steps take
+// their 16 rows from wherever they are.
+// Roles: warps 0-3 and 4-7 are two softmax warpgroups that alternate sub-tiles, each with its own Q buffer and its
+// own 256 TMEM columns (S in [0, 144), P over its first 72 columns, O in [128, 256)); warp 8 issues the TMA loads,
+// warp 9 the S MMAs, warp 11 the PV MMAs, warp 10 the TMA stores of staged output tiles.  All of them count
+// sub-tiles with one per-block counter g, so the Q load, the S MMA, the softmax, the PV MMA and the store of
+// neighbouring sub-tiles overlap.
+namespace stream {
 constexpr int SUB = 16;                         // tokens per sub-tile
-constexpr int NSUB = 8;                         // sub-tiles per block
-constexpr int N = 144;                          // keys per sub-tile (16 + 127, rounded up to 16)
+constexpr int N = 144;                          // keys per sub-tile
 constexpr int KV_ROWS = 256;
 constexpr int KV_HALF = KV_ROWS * 128;          // bytes of one 64-element half
 constexpr int KV_BYTES = 2 * KV_HALF;           // 64 KB
 constexpr int QBUF = 2;                         // Q tiles in flight (a buffer is free as soon as its S MMA has run)
 constexpr int OFF_Q = 0, OFF_K = QBUF * TILE_BYTES, OFF_V = OFF_K + KV_BYTES, OFF_STAGE = OFF_V + KV_BYTES;
 constexpr int SMEM = OFF_STAGE + TILE_BYTES + 1024;   // 225 KB: Q 64, K 64, V 64, output staging 32
-constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-enum { B_K = 0, B_V = 1, B_QFULL = 2, B_QEMPTY = 4, B_SFULL = 6, B_PFULL = 8, B_OFULL = 10, B_OFREE = 12, B_STAGED = 14,
-       B_STGFREE = 15, NBARS = 16 };
-constexpr int THREADS = 352;                    // 8 softmax warps + producer + MMA issuer + output store warp
-}  // namespace pipe
+constexpr int SLOTS = 16;
+constexpr int THREADS = 384;  // 8 softmax warps + producer + S issuer + output store warp + PV issuer
+// Registers per thread after the roles have split (the launch gives every thread the same number; a request for
+// more blocks until other warps of the block have given theirs up, so the sum must not pass what the launch gave:
+// checked against the compiled kernel before every launch)
+constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 224;
+enum { B_QFULL = 0, B_QEMPTY = 2, B_SFULL = 4, B_PFULL = 6, B_OFULL = 8, B_OFREE = 10, B_STAGED = 12, B_STGFREE = 13,
+       B_PHALF = 14 /* the first 64 keys of P posted */, B_DRAIN = 16 /* every MMA of a finished stream has run */,
+       B_KP = 17, B_VP = 17 + SLOTS, NBARS = 17 + 2 * SLOTS };
+// instruction descriptor of an S MMA over n keys (a multiple of 16)
+__device__ __forceinline__ uint32_t idesc_s(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+// The sub-tiles a block walks: units [u, u_end) of the flattened (stream, sub-tile) space, empty ones skipped.
+struct Walker {
+  const int32_t* q_indptr;
+  int Hkv, ns_max, u, u_end, st, sidx, cur_stream, r_cur, kh_cur, t0, n, ns;
+  bool fresh;  // the sub-tile returned last is the first this block takes from its stream
+  __device__ Walker(const PrefillParams& p_, int ns_max_, int u0, int u1)
+      : q_indptr(p_.b.q_indptr), Hkv(p_.m.Hkv), ns_max(ns_max_), u(u0), u_end(u1), st(u0 / ns_max_), sidx(u0 % ns_max_),
+        cur_stream(-1), r_cur(0), kh_cur(0), t0(0), n(0), ns(0), fresh(false) {}
+  // next non-empty sub-tile: request r, KV head kh, first chunk-relative token i; false when the range is used up
+  __device__ bool next(int& r, int& kh, int& i) {
+    while (u < u_end) {
+      bool changed = false;
+      if (st != cur_stream) {
+        cur_stream = st;
+        r_cur = st / Hkv;
+        kh_cur = st - r_cur * Hkv;
+        t0 = q_indptr[r_cur];
+        n = q_indptr[r_cur + 1] - t0;
+        ns = n > 128 ? (n - 128 + SUB - 1) / SUB : 0;
+        changed = true;
+      }
+      if (sidx >= ns) {  // nothing (left) in this stream: jump to the next one
+        u += ns_max - sidx;
+        ++st;
+        sidx = 0;
+        continue;
+      }
+      r = r_cur;
+      kh = kh_cur;
+      i = 128 + sidx * SUB;
+      fresh = changed;
+      ++u;
+      if (++sidx == ns_max) {
+        ++st;
+        sidx = 0;
+      }
+      return true;
+    }
+    return false;
+  }
+};
+// Number of non-empty sub-tiles among units [u0, u1).
+__device__ inline int count_sub_tiles(const PrefillParams& p, int ns_max, int u0, int u1) {
+  int total = 0;
+  for (int st = u0 / ns_max; st * ns_max < u1; ++st) {
+    const int r = st / p.m.Hkv, n = p.b.q_indptr[r + 1] - p.b.q_indptr[r];
+    const int ns = n > 128 ? (n - 128 + SUB - 1) / SUB : 0;
+    const int lo = max(u0, st * ns_max), hi = min(u1, st * ns_max + ns);
+    total += max(0, hi - lo);
+  }
+  return total;
+}
+}  // namespace stream
 
-__global__ void __launch_bounds__(pipe::THREADS, 1)
-prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_out,
-                        const PrefillParams p, const int first_block, const int tma_out) {
-  using pipe::SUB; using pipe::NSUB; using pipe::N; using pipe::KV_HALF; using pipe::KV_BYTES;
-  using pipe::B_K; using pipe::B_V; using pipe::B_QFULL; using pipe::B_QEMPTY; using pipe::B_SFULL; using pipe::B_PFULL;
-  using pipe::B_OFULL; using pipe::B_OFREE; using pipe::B_STAGED; using pipe::B_STGFREE; using pipe::NBARS; using pipe::QBUF;
+__global__ void __launch_bounds__(stream::THREADS, 1)
+prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k16,
+                          const __grid_constant__ CUtensorMap tm_v16, const __grid_constant__ CUtensorMap tm_out,
+                          const PrefillParams p, const int ns_max, const int units_per_block, const int tma_out) {
+  using namespace stream;
   constexpr int G = 8;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[NBARS];
   __shared__ uint32_t tmem_base_slot;
+  // what the softmax warps need to know about a sub-tile, written by the producer when it issues the Q load:
+  // {first token (row of q / out), valid tokens, KV head, index among the staged tiles or -1}
+  __shared__ int4 tile_info[4];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
-
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kh = blockIdx.x, r = blockIdx.z;
-  const int t0 = p.b.q_indptr[r];
-  const int n = p.b.q_indptr[r + 1] - t0;
-  const int i0 = (first_block + (int)blockIdx.y) * 128;  // first chunk-relative token of this block (>= 128)
-  if (i0 >= n) return;
+  const int total_units = p.b.B * M.Hkv * ns_max;
+  const int u0 = blockIdx.x * units_per_block, u1 = min(u0 + units_per_block, total_units);
+  if (u0 >= u1) return;
   if (*reinterpret_cast<volatile int32_t*>(p.err) != 0) return;
-  const int n_sub = min(NSUB, (n - i0 + SUB - 1) / SUB);
-  const int key0 = i0 - 128;  // chunk-relative index of row 0 of the K/V buffer
 
   auto bar = [&](int i) { return smem_u32(&bars[i]); };
   if (threadIdx.x == 0) {
-    mbar_init(bar(B_K), 1);
-    mbar_init(bar(B_V), 1);
     mbar_init(bar(B_STAGED), 4);
     mbar_init(bar(B_STGFREE), 1);
+    mbar_init(bar(B_DRAIN), 1);
     for (int q = 0; q < QBUF; ++q) {
       mbar_init(bar(B_QFULL + q), 1);
       mbar_init(bar(B_QEMPTY + q), 1);
@@ -1077,8 +1139,13 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     for (int u = 0; u < 2; ++u) {
       mbar_init(bar(B_SFULL + u), 1);
       mbar_init(bar(B_PFULL + u), 4);
+      mbar_init(bar(B_PHALF + u), 4);
       mbar_init(bar(B_OFULL + u), 1);
       mbar_init(bar(B_OFREE + u), 4);
+    }
+    for (int j = 0; j < SLOTS; ++j) {
+      mbar_init(bar(B_KP + j), 1);
+      mbar_init(bar(B_VP + j), 1);
     }
     mbar_fence_init();
   }
@@ -1092,122 +1159,198 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
+  // Registers move from the four service warps (one warpgroup) to the two softmax warpgroups, whose threads hold a
+  // whole row of 144 scores plus its exponentials' state: 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168.
+  // (each role's branch changes its own allotment: the compiler budgets a branch by the instruction that dominates it)
   if (warp == 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
     // ======================= TMA producer =======================
     if (lane == 0) {
-      mbar_arrive_expect_tx(bar(B_K), KV_BYTES);
-      for (int hf = 0; hf < 2; ++hf)
-        for (int rb = 0; rb < 2; ++rb)
-          tma_load_3d(sbase + pipe::OFF_K + hf * KV_HALF + rb * 128 * 128, &tm_k, bar(B_K), hf * 64, kh, t0 + key0 + rb * 128);
+      Walker w(p, ns_max, u0, u1);
+      int r, kh, i, n_staged = 0, n_switch = 0;
       bool ok = true;
-      for (int s = 0; s < n_sub && ok; ++s) {
-        const int qb = s % QBUF;
-        if (s >= QBUF && !mbar_wait(bar(B_QEMPTY + qb), ((s / QBUF) - 1) & 1)) {
-          record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 60);
+      // one 16-key piece (keys [key, key + 16) of the chunk) of K and of V into its slot
+      auto load_piece = [&](int t0, int kh_, int key) {
+        const int slot = (key / SUB) % SLOTS;
+        mbar_arrive_expect_tx(bar(B_KP + slot), 2 * SUB * 128);
+        mbar_arrive_expect_tx(bar(B_VP + slot), 2 * SUB * 128);
+        for (int hf = 0; hf < 2; ++hf) {
+          tma_load_3d(sbase + stream::OFF_K + hf * KV_HALF + slot * SUB * 128, &tm_k16, bar(B_KP + slot), hf * 64, kh_, t0 + key);
+          tma_load_3d(sbase + stream::OFF_V + hf * KV_HALF + slot * SUB * 128, &tm_v16, bar(B_VP + slot), hf * 64, kh_, t0 + key);
+        }
+      };
+      for (int g = 0; ok && w.next(r, kh, i); ++g) {
+        const int qb = g % QBUF;
+        // Q buffer qb is free once S(g - 2) has run; in-order MMA execution then also has S(g - 8) and PV(g - 8)
+        // behind it, which were the last readers of the slot this sub-tile's piece goes to
+        if (g >= QBUF && !mbar_wait(bar(B_QEMPTY + qb), ((g / QBUF) - 1) & 1)) {
+          record_error(p.err, HSWA_ERR_TIMEOUT, r, g, 70);
           ok = false;
           break;
         }
+        if (w.fresh) {
+          // a new stream: its first eight pieces go to slots the previous stream's last sub-tiles may still be reading.
+          // The PV issuer commits to a barrier of its own at every such switch, so this thread sees each of that
+          // barrier's phases in turn.  (The per-sub-tile barriers will not do: a parity wait tells a phase only from its
+          // neighbours, and this thread may be one phase behind or two ahead of them.)
+          if (g > 0 && !mbar_wait(bar(B_DRAIN), n_switch++ & 1)) {
+            record_error(p.err, HSWA_ERR_TIMEOUT, r, g, 71);
+            ok = false;
+            break;
+          }
+          for (int key = i - 128; key < i; key += SUB) load_piece(w.t0, kh, key);
+        }
+        // entry g & 3 was last read for sub-tile g - 4, whose accumulator S(g - 2) has waited for
+        {
+          const bool staged_tile = tma_out && i + SUB <= w.n;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(&tile_info[g & 3])), "r"(w.t0 + i),
+                       "r"(min(SUB, w.n - i)), "r"(kh), "r"(staged_tile ? n_staged : -1)
+                       : "memory");
+          if (staged_tile) ++n_staged;
+          __threadfence_block();
+        }
         mbar_arrive_expect_tx(bar(B_QFULL + qb), TILE_BYTES);
         for (int hf = 0; hf < 2; ++hf)
-          tma_load_3d(sbase + pipe::OFF_Q + qb * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(B_QFULL + qb), hf * 64, kh * G, t0 + i0 + s * SUB);
-        if (s == 1 || n_sub == 1) {  // V is needed after the first softmax only: queue it behind the first Q tiles
-          mbar_arrive_expect_tx(bar(B_V), KV_BYTES);
-          for (int hf = 0; hf < 2; ++hf)
-            for (int rb = 0; rb < 2; ++rb)
-              tma_load_3d(sbase + pipe::OFF_V + hf * KV_HALF + rb * 128 * 128, &tm_v, bar(B_V), hf * 64, kh, t0 + key0 + rb * 128);
-        }
+          tma_load_3d(sbase + stream::OFF_Q + qb * TILE_BYTES + hf * HALF_BYTES, &tm_q, bar(B_QFULL + qb), hf * 64, kh * G, w.t0 + i);
+        load_piece(w.t0, kh, i);
       }
     }
   } else if (warp == 9) {
-    // ======================= MMA issuer =======================
-    if (lane == 0) {
-      auto issue_S = [&](int s) {
-        const int u = s & 1;
-        tc_fence_after();
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
+    // ======================= MMA issuers =======================
+    // Warp 9 issues the S MMAs, warp 11 the PV MMAs.  Each has one chain of barriers to wait for, in order, so it can
+    // sleep in the wait; a single thread that polls both chains in turn spends more time polling (a test of a
+    // completed mbarrier costs 100-250 clocks while the tensor cores use shared memory) than issuing.  The whole
+    // warp walks the loop converged (waits, descriptor arithmetic); one elected lane issues.  Descriptors are
+    // built once and advanced by additions.  The tensor pipe runs the two warps' MMAs in the order they arrive;
+    // every dependence between them goes through a barrier (P posted, accumulator read out).
+    Walker w(p, ns_max, u0, u1);
+    uint32_t par = 0;  // per slot: parity of the fill to wait for next
+    int r, kh, i;
+    bool ok = true;
+    const uint64_t dQ0 = smem_desc(sbase + stream::OFF_Q, 16), dQ1 = smem_desc(sbase + stream::OFF_Q + TILE_BYTES, 16);
+    const uint64_t dK0 = smem_desc(sbase + stream::OFF_K, 16);
+    auto wait_piece = [&](int key) {
+      const int slot = (key / SUB) % SLOTS;
+      const bool got = mbar_wait(bar(B_KP + slot), (par >> slot) & 1u);
+      par ^= 1u << slot;
+      return got;
+    };
+    for (int g = 0; ok && w.next(r, kh, i); ++g) {
+      const int u = g & 1, start = (i - 128) & (SLOTS * SUB - 1);  // first row of the slice in the circular buffer
+      const int n1 = min(N, SLOTS * SUB - start), n2 = N - n1;
+      const uint64_t dq = (g % QBUF) ? dQ1 : dQ0, dk = desc_advance(dK0, start * 128);
+      const uint32_t id1 = idesc_s(n1), id2 = idesc_s(n2);
+      // the accumulator of sub-tile g - 2 read out, Q(g) in shared memory, the keys: this sub-tile's own piece and,
+      // for the first sub-tile of a stream, the eight before it
+      if (g >= 2) ok = mbar_wait(bar(B_OFREE + u), ((g >> 1) - 1) & 1);
+      if (ok) ok = mbar_wait(bar(B_QFULL + g % QBUF), (g / QBUF) & 1);
+      if (w.fresh)
+        for (int key = i - 128; key < i && ok; key += SUB) ok = wait_piece(key);
+      if (ok) ok = wait_piece(i);
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t aq = sbase + pipe::OFF_Q + (s % QBUF) * TILE_BYTES + (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-          const uint32_t ak = sbase + pipe::OFF_K + (ks >> 2) * KV_HALF + s * SUB * 128 + (ks & 3) * 32;
-          tc_mma_ss(tmem + u * 256, smem_desc(aq, 16), smem_desc(ak, 16), pipe::IDESC_S, ks > 0);
+        for (int ks = 0; ks < HD / 16; ++ks)
+          tc_mma_ss(tmem + u * 256, desc_advance(dq, (ks >> 2) * HALF_BYTES + (ks & 3) * 32),
+                    desc_advance(dk, (ks >> 2) * KV_HALF + (ks & 3) * 32), id1, ks > 0);
+        if (n2 > 0) {  // the slice wraps: its last n2 keys are the buffer's first rows
+#pragma unroll
+          for (int ks = 0; ks < HD / 16; ++ks)
+            tc_mma_ss(tmem + u * 256 + n1, desc_advance(dq, (ks >> 2) * HALF_BYTES + (ks & 3) * 32),
+                      desc_advance(dK0, (ks >> 2) * KV_HALF + (ks & 3) * 32), id2, ks > 0);
         }
         tc_commit(bar(B_SFULL + u));
-        tc_commit(bar(B_QEMPTY + s % QBUF));  // Q(s) has been consumed once these MMAs are done
-      };
-      auto issue_PV = [&](int s) {
-        const int u = s & 1;
-        tc_fence_after();
+        tc_commit(bar(B_QEMPTY + g % QBUF));  // Q(g) has been consumed once these MMAs are done
+      }
+      __syncwarp();
+    }
+    if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, 0, 72);
+  } else if (warp == 11) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
+    Walker w(p, ns_max, u0, u1);
+    uint32_t par = 0;
+    int r, kh, i;
+    bool ok = true;
+    const uint64_t dV0 = smem_desc(sbase + stream::OFF_V, KV_HALF);
+    auto wait_piece = [&](int key) {
+      const int slot = (key / SUB) % SLOTS;
+      const bool got = mbar_wait(bar(B_VP + slot), (par >> slot) & 1u);
+      par ^= 1u << slot;
+      return got;
+    };
+    for (int g = 0; ok && w.next(r, kh, i); ++g) {
+      const int u = g & 1, start = (i - 128) & (SLOTS * SUB - 1);
+      if (w.fresh) {
+        if (g > 0) {  // every MMA of the stream that has just ended: the producer waits for this before it reuses slots
+          if (elect_one()) tc_commit(bar(B_DRAIN));
+          __syncwarp();
+        }
+        for (int key = i - 128; key < i && ok; key += SUB) ok = wait_piece(key);
+      }
+      // the first 64 keys of P are posted while the rest of the row's exponentials run
+      if (ok) ok = mbar_wait(bar(B_PHALF + u), (g >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) {
 #pragma unroll
-        for (int kk = 0; kk < N / 16; ++kk)
-          tc_mma_ts(tmem + u * 256 + 128, tmem + u * 256 + kk * 8, smem_desc(sbase + pipe::OFF_V + s * SUB * 128 + kk * 2048, KV_HALF),
-                    IDESC_PV, kk > 0);
-        tc_commit(bar(B_OFULL + u));
-      };
-      // Issue whichever MMA group has its inputs first: S(s) needs Q(s) in shared memory and, from the third
-      // sub-tile on, the output of S(s - 2)'s TMEM buffer read out; PV(s) needs P(s) (and V).  Sub-tiles of the
-      // two warpgroups interleave, so neither waits behind the other's hand-off.
-      bool ok = mbar_wait(bar(B_K), 0);
-      int next_s = 0, next_pv = 0;
-      bool v_ready = false;
-      long long t_start = clock64();
-      while (ok && next_pv < n_sub) {
-        bool progress = false;
-        if (next_s < n_sub) {
-          const int s = next_s;
-          const bool free_ok = s < 2 || mbar_try_wait(bar(B_OFREE + (s & 1)), ((s >> 1) - 1) & 1);
-          if (free_ok && mbar_try_wait(bar(B_QFULL + s % QBUF), (s / QBUF) & 1)) {
-            issue_S(s);
-            ++next_s;
-            progress = true;
-          }
-        }
-        if (next_pv < next_s && mbar_try_wait(bar(B_PFULL + (next_pv & 1)), (next_pv >> 1) & 1)) {
-          if (!v_ready) {
-            ok = mbar_wait(bar(B_V), 0);
-            v_ready = true;
-          }
-          if (ok) issue_PV(next_pv);
-          ++next_pv;
-          progress = true;
-        }
-        if (progress) {
-          t_start = clock64();
-        } else if (clock64() - t_start > 4000000000LL) {
-          ok = false;
+        for (int kk = 0; kk < 4; ++kk) {
+          const int row = (start + kk * 16) & (SLOTS * SUB - 1);
+          tc_mma_ts(tmem + u * 256 + 128, tmem + u * 256 + kk * 8, desc_advance(dV0, row * 128), IDESC_PV, kk > 0);
         }
       }
-      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 61);
+      __syncwarp();
+      ok = wait_piece(i);
+      if (ok) ok = mbar_wait(bar(B_PFULL + u), (g >> 1) & 1);
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) {
+#pragma unroll
+        for (int kk = 4; kk < N / 16; ++kk) {
+          const int row = (start + kk * 16) & (SLOTS * SUB - 1);
+          tc_mma_ts(tmem + u * 256 + 128, tmem + u * 256 + kk * 8, desc_advance(dV0, row * 128), IDESC_PV, 1u);
+        }
+        tc_commit(bar(B_OFULL + u));
+      }
+      __syncwarp();
     }
+    if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, 1, 72);
   } else if (warp == 10) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
     // ======================= output store warp =======================
-    // Takes each staged output tile to global memory with one TMA tensor store per half and frees the staging
-    // buffer once shared memory has been read, so no softmax thread waits for a store.
     if (lane == 0 && tma_out) {
+      Walker w(p, ns_max, u0, u1);
+      int r, kh, i, n_staged = 0;
       bool ok = true;
-      for (int s = 0; s < n_sub && ok; ++s) {
-        if (i0 + s * SUB + SUB > n) break;  // a ragged last sub-tile is stored directly by its warpgroup
-        ok = mbar_wait(bar(B_STAGED), s & 1);
+      for (int g = 0; ok && w.next(r, kh, i); ++g) {
+        if (i + SUB > w.n) continue;  // a ragged last sub-tile is stored directly by its warpgroup
+        ok = mbar_wait(bar(B_STAGED), n_staged & 1);
         if (!ok) break;
         for (int hf = 0; hf < 2; ++hf)
           asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(&tm_out),
-                       "r"(sbase + pipe::OFF_STAGE + hf * HALF_BYTES), "r"(hf * 64), "r"(kh * G), "r"(t0 + i0 + s * SUB)
+                       "r"(sbase + stream::OFF_STAGE + hf * HALF_BYTES), "r"(hf * 64), "r"(kh * G), "r"(w.t0 + i)
                        : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory has been read
         mbar_arrive(bar(B_STGFREE));
+        ++n_staged;
       }
-      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, r, i0, 63);
+      if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, n_staged, 73);
       asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // stores have landed
     }
   } else {
     // ======================= softmax warpgroups: warps 0-3 take even sub-tiles, 4-7 odd =======================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX) : "memory");
     const int u = warp >> 2;
     const int rr = (warp & 3) * 32 + lane;  // row = TMEM lane
-    const int tl = rr / G, g = rr % G;      // token within the sub-tile, head within the group
+    const int tl = rr / G, gh = rr % G;     // token within the sub-tile, head within the group
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_addr + u * 256, tO = tS + 128;
     const int lo = tl + 129 - M.W, hi = tl + 129;  // visible key columns [lo, hi) of the 144-key slice
-    for (int s = u; s < n_sub; s += 2) {
-      const uint32_t par = (s >> 1) & 1;
+    const int n_total = count_sub_tiles(p, ns_max, u0, u1);
+    for (int g = u; g < n_total; g += 2) {
+      const uint32_t par = (g >> 1) & 1;
       bool ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SFULL + u), par));
       float l_run = 0.f, m_use = 0.f;
       if (ok) {
@@ -1245,79 +1388,92 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         float2 acc[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[c] = make_float2(0.f, 0.f);
+        auto exps = [&](int k0, int k1) {
 #pragma unroll
-        for (int k = 0; k < N / 2; ++k) {
-          const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
-          const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));  // masked columns: 2^(-inf) = 0
-          v[k] = pack_bf16x2(e.x, e.y);
-          // the row sum takes the fp32 values before their rounding to bf16 (summing the rounded ones instead
-          // costs one more ALU op per key and 7-8 % of the kernel's time; the difference shows only for nearly
-          // one-hot rows, where it is bounded by 2^-9 max|v|)
-          acc[k & 3] = __fadd2_rn(acc[k & 3], e);
-        }
+          for (int k = k0; k < k1; ++k) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1])), sc2, nm2);
+            const float2 e = make_float2(fast_exp2(x.x), fast_exp2(x.y));  // masked columns: 2^(-inf) = 0
+            v[k] = pack_bf16x2(e.x, e.y);
+            acc[k & 3] = __fadd2_rn(acc[k & 3], e);  // row sum of the fp32 values, not of the rounded ones
+          }
+        };
+        // P of the first 64 keys is stored while the next exponentials run and posted on its own, so that the PV
+        // MMAs of those keys run under the rest of the row
+        exps(0, 32);
+        tmem_st32(tS, v);
+        exps(32, 44);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_PHALF + u));
+        exps(44, N / 2);
         const float2 a01 = __fadd2_rn(acc[0], acc[1]), a23 = __fadd2_rn(acc[2], acc[3]);
         l_run = (a01.x + a01.y) + (a23.x + a23.y);
-        tmem_st32(tS, v);
         tmem_st32(tS + 32, v + 32);
         tmem_st8(tS + 64, v + 64);
         tc_wait_st();
-      } else if (lane == 0) {
-        record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 62);
+      } else {
+        if (lane == 0) {
+          record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, g, 74);
+          mbar_arrive(bar(B_PHALF + u));
+        }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_PFULL + u));
       if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OFULL + u), par));
       tc_fence_after();
+      // (the producer wrote the entry before it issued this sub-tile's Q load, which S(g) has consumed)
+      int4 info;
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(info.x), "=r"(info.y), "=r"(info.z), "=r"(info.w)
+                   : "r"(smem_u32(&tile_info[g & 3]))
+                   : "memory");
+      const int my_stage_idx = info.w;
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      const int tok = i0 + s * SUB + tl;
-      const bool row_ok = ok && tok < n;
-      const int64_t orow = (int64_t)(t0 + tok) * M.Hq + kh * G + g;
-      // Full sub-tiles with bf16 output leave through a shared-memory staging tile and one TMA tensor store; a row-per-thread global store would touch 32 scattered sectors per
-      // instruction.  Ragged tails and fp32 output use plain stores.
-      const bool staged = tma_out && ok && (i0 + s * SUB + SUB <= n);
-      uint8_t* stage = smem + pipe::OFF_STAGE;
+      const bool row_ok = ok && tl < info.y;
+      const int64_t orow = (int64_t)(info.x + tl) * M.Hq + info.z * G + gh;
+      const bool staged = my_stage_idx >= 0 && ok;
+      uint8_t* stage = smem + stream::OFF_STAGE;
       {
-        uint32_t w[128];  // the whole accumulator row in one round trip
-        tmem_ld32(tO, w);
-        tmem_ld32(tO + 32, w + 32);
-        tmem_ld32(tO + 64, w + 64);
-        tmem_ld32(tO + 96, w + 96);
+        uint32_t wv[128];  // the whole accumulator row in one round trip
+        tmem_ld32(tO, wv);
+        tmem_ld32(tO + 32, wv + 32);
+        tmem_ld32(tO + 64, wv + 64);
+        tmem_ld32(tO + 96, wv + 96);
         tc_wait_ld();
         // the accumulator has been read out: the MMA warp may reuse this TMEM buffer
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(B_OFREE + u));
         if (staged) {
-          // sub-tiles use the single staging tile in order: wait until the previous one's store has read it
-          if (s > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(B_STGFREE), (s - 1) & 1))) {
-            if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, s, 64);
+          // staged sub-tiles use the single staging tile in order: wait until the previous one's store has read it
+          // (the row is scaled and packed first: that work needs no staging tile)
+#pragma unroll
+          for (int c = 0; c < 64; ++c) wv[c] = pack_bf16x2(__uint_as_float(wv[2 * c]) * inv, __uint_as_float(wv[2 * c + 1]) * inv);
+          if (my_stage_idx > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(B_STGFREE), (my_stage_idx - 1) & 1))) {
+            if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, g, 75);
           }
 #pragma unroll
-          for (int chunk = 0; chunk < 16; ++chunk) {  // 16-byte chunks of the 256-byte bf16 row
-            uint4 x;
-            x.x = pack_bf16x2(__uint_as_float(w[8 * chunk]) * inv, __uint_as_float(w[8 * chunk + 1]) * inv);
-            x.y = pack_bf16x2(__uint_as_float(w[8 * chunk + 2]) * inv, __uint_as_float(w[8 * chunk + 3]) * inv);
-            x.z = pack_bf16x2(__uint_as_float(w[8 * chunk + 4]) * inv, __uint_as_float(w[8 * chunk + 5]) * inv);
-            x.w = pack_bf16x2(__uint_as_float(w[8 * chunk + 6]) * inv, __uint_as_float(w[8 * chunk + 7]) * inv);
-            *reinterpret_cast<uint4*>(stage + (chunk >> 3) * HALF_BYTES + swz128(rr, chunk & 7)) = x;
-          }
+          for (int chunk = 0; chunk < 16; ++chunk)  // 16-byte chunks of the 256-byte bf16 row
+            *reinterpret_cast<uint4*>(stage + (chunk >> 3) * HALF_BYTES + swz128(rr, chunk & 7)) =
+                make_uint4(wv[4 * chunk], wv[4 * chunk + 1], wv[4 * chunk + 2], wv[4 * chunk + 3]);
         } else if (row_ok) {
           if (M.out_fp32) {
             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + orow * HD);
 #pragma unroll
             for (int k = 0; k < 32; ++k)
-              dst[k] = make_float4(__uint_as_float(w[4 * k]) * inv, __uint_as_float(w[4 * k + 1]) * inv,
-                                   __uint_as_float(w[4 * k + 2]) * inv, __uint_as_float(w[4 * k + 3]) * inv);
+              dst[k] = make_float4(__uint_as_float(wv[4 * k]) * inv, __uint_as_float(wv[4 * k + 1]) * inv,
+                                   __uint_as_float(wv[4 * k + 2]) * inv, __uint_as_float(wv[4 * k + 3]) * inv);
           } else {
             uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + orow * HD);
 #pragma unroll
             for (int k = 0; k < 16; ++k) {
               uint4 x;
-              x.x = pack_bf16x2(__uint_as_float(w[8 * k]) * inv, __uint_as_float(w[8 * k + 1]) * inv);
-              x.y = pack_bf16x2(__uint_as_float(w[8 * k + 2]) * inv, __uint_as_float(w[8 * k + 3]) * inv);
-              x.z = pack_bf16x2(__uint_as_float(w[8 * k + 4]) * inv, __uint_as_float(w[8 * k + 5]) * inv);
-              x.w = pack_bf16x2(__uint_as_float(w[8 * k + 6]) * inv, __uint_as_float(w[8 * k + 7]) * inv);
+              x.x = pack_bf16x2(__uint_as_float(wv[8 * k]) * inv, __uint_as_float(wv[8 * k + 1]) * inv);
+              x.y = pack_bf16x2(__uint_as_float(wv[8 * k + 2]) * inv, __uint_as_float(wv[8 * k + 3]) * inv);
+              x.z = pack_bf16x2(__uint_as_float(wv[8 * k + 4]) * inv, __uint_as_float(wv[8 * k + 5]) * inv);
+              x.w = pack_bf16x2(__uint_as_float(wv[8 * k + 6]) * inv, __uint_as_float(wv[8 * k + 7]) * inv);
               dst[k] = x;
             }
           }
@@ -1340,14 +1496,25 @@ prefill_swa_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   }
 }
 
-cudaError_t launch_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_out,
-                        int tma_out, const PrefillParams& p, int first_block, cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(prefill_swa_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe::SMEM);
+cudaError_t launch_stream(const CUtensorMap& tm_q, const CUtensorMap& tm_k16, const CUtensorMap& tm_v16, const CUtensorMap& tm_out,
+                          int tma_out, const PrefillParams& p, int num_sms, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(prefill_swa_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM);
   if (e != cudaSuccess) return e;
-  const int blocks = (p.max_q_len + 127) / 128 - first_block;
-  if (blocks <= 0) return cudaSuccess;
-  dim3 grid(p.m.Hkv, blocks, p.b.B);
-  prefill_swa_pipe_kernel<<<grid, pipe::THREADS, pipe::SMEM, s>>>(tm_q, tm_k, tm_v, tm_out, p, first_block, tma_out);
+  static int regs_at_launch = 0;
+  if (regs_at_launch == 0) {
+    cudaFuncAttributes attr;
+    e = cudaFuncGetAttributes(&attr, prefill_swa_stream_kernel);
+    if (e != cudaSuccess) return e;
+    regs_at_launch = attr.numRegs;
+  }
+  // the softmax warps' request for registers would never be granted
+  if (regs_at_launch * stream::THREADS < 128 * stream::REGS_SERVICE + 256 * stream::REGS_SOFTMAX) return cudaErrorLaunchOutOfResources;
+  const int ns_max = (p.max_q_len - 128 + stream::SUB - 1) / stream::SUB;
+  if (ns_max <= 0) return cudaSuccess;
+  const long long units = (long long)p.b.B * p.m.Hkv * ns_max;
+  const int blocks = (int)(units < num_sms ? units : num_sms);
+  const int per = (int)((units + blocks - 1) / blocks);
+  prefill_swa_stream_kernel<<<blocks, stream::THREADS, stream::SMEM, s>>>(tm_q, tm_k16, tm_v16, tm_out, p, ns_max, per, tma_out);
   return cudaGetLastError();
 }
 
@@ -1369,17 +1536,6 @@ cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtens
   if (p.m.G == 8) return launch_packed<8>(tm_q, tm_k, tm_v, p, first_tok, s);
   if (p.m.G == 4) return launch_packed<4>(tm_q, tm_k, tm_v, p, first_tok, s);
   return cudaErrorInvalidValue;
-}
-
-// Pipelined SWA kernel (GQA group of 8): blocks of 128 tokens starting at block `first_block`; tm_q has box
-// {64, 8 heads, 16 tokens}, tm_k / tm_v have box {64, 1, 128 rows}; tm_out is tm_q's twin over a bf16 output
-// tensor (used when tma_out != 0).
-cudaError_t hswa_launch_prefill_swa_pipe(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                         const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int first_block,
-                                         cudaStream_t s) {
-  if (p.m.G != 8) return cudaErrorInvalidValue;
-  if (p.b.B == 0) return cudaSuccess;
-  return launch_pipe(tm_q, tm_k, tm_v, tm_out, tma_out, p, first_block, s);
 }
 
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
@@ -1405,4 +1561,13 @@ cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensor
   dim3 grid(n_slices, p.m.Hkv, (p.b.B + 31) / 32);
   prefill_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_pool, tm_pool, p, 1);
   return cudaGetLastError();
+}
+
+// Streaming SWA kernel (GQA group of 8, window 128): every token from the 129th of each request on.  tm_q has box
+// {64, 8 heads, 16 tokens}, tm_k16 / tm_v16 have box {64, 1, 16 rows}; tm_out is tm_q's twin over a bf16 output
+// tensor (used when tma_out != 0).
+cudaError_t hswa_launch_prefill_swa_stream(const CUtensorMap& tm_q, const CUtensorMap& tm_k16, const CUtensorMap& tm_v16,
+                                           const CUtensorMap& tm_out, int tma_out, const PrefillParams& p, int num_sms,
+                                           cudaStream_t s) {
+  return launch_stream(tm_q, tm_k16, tm_v16, tm_out, tma_out, p, num_sms, s);
 }

@@ -432,7 +432,7 @@ def test_prefill_tc_sweep(d, is_swa):
 @pytest.mark.parametrize("W", [64, 96, 33])
 @pytest.mark.parametrize("G", [8, 4, 2])
 def test_prefill_tc_other_windows(W, G):
-    """Windows other than the paper's 128: the pipelined SWA kernel is bypassed and the packed / tile kernels
+    """Windows other than the paper's 128: the streaming SWA kernel is bypassed and the packed / tile kernels
     must apply the general window mask."""
     d = dims(G, 128, 64, 1, W=W)
     ctx = [0, 1, W - 1, W, 200, 64]
@@ -452,6 +452,34 @@ def test_prefill_tc_long_context_and_many_requests():
     for is_swa in (False, True):
         err, lerr = run_prefill(sc, is_swa)
         assert err <= TOL and lerr <= TOL, (is_swa, err, lerr)
+
+
+@pytest.mark.parametrize("case", ["many_short_streams", "one_long_stream", "two_long_streams", "fewer_units_than_sms"])
+def test_prefill_swa_stream_walk(case):
+    """The streaming SWA kernel (group of 8, W = 128) hands each persistent block a run of 16-token sub-tiles that may
+    begin in the middle of one (request, KV head) stream, skip streams that have no token past the 128th, and end in
+    another stream: mixes of chunk lengths that put several stream switches, many empty streams, or a single
+    sub-tile into one block's run, with ragged last sub-tiles, against the oracle in both output types."""
+    rng = np.random.default_rng(61)
+    if case == "many_short_streams":      # one long request sets the stride of the unit space; the rest own 0-3 sub-tiles
+        d = dims(8, 128, 64, 2)
+        q_len = [3001] + [int(x) for x in rng.integers(100, 180, 63)]
+    elif case == "one_long_stream":       # every block starts and ends inside the same stream
+        d = dims(8, 128, 64, 1)
+        q_len = [128 + 16 * 148 * 3 + 5]
+    elif case == "two_long_streams":      # blocks in the middle of the grid cross from one KV head / request to the next
+        d = dims(8, 128, 64, 2)
+        q_len = [128 + 16 * 203 + 9, 128 + 16 * 77 + 16]
+    else:                                 # fewer sub-tiles than SMs: one unit per block
+        d = dims(8, 128, 64, 1)
+        q_len = [129, 160, 145, 128, 7]
+    ctx = [int(x) for x in rng.integers(0, 300, len(q_len))]
+    sc = build_scenario(d, ctx, q_len, seed=62)
+    got32, ref, lerr = run_prefill(sc, True, arrays=True)
+    assert np.abs(got32 - ref).max() <= TOL and lerr <= TOL, (np.abs(got32 - ref).max(), lerr)
+    got16, _, _ = run_prefill(sc, True, fuse_append=False, out_dtype=torch.bfloat16, arrays=True)
+    want16 = torch.from_numpy(got32.astype(np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
+    assert np.array_equal(got16, want16)
 
 
 # ---------------------------------------------------------------------------------------------------------
