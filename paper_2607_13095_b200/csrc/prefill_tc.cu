@@ -34,7 +34,10 @@ constexpr int PG = 64;                // page size
 constexpr int HALF_BYTES = 128 * 128; // [128 rows][128 B]: one 64-element half of a 128-row tile
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int KV_STAGES = 2;
-constexpr int NUM_THREADS = 352;  // 8 softmax warps + producer + one MMA issuer per Q tile
+constexpr int NUM_THREADS = 384;  // 8 softmax warps + producer + one MMA issuer per Q tile + an idle warp (see the kernel)
+// Registers per thread after the roles have split; the sum over the block must not pass what the launch gave
+// (384 x 168), or the softmax warps' request would never be granted: checked against the compiled kernel before launch.
+constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 224;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                  // 2 Q tiles
@@ -422,7 +425,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
+  // Registers move from the service warps (one warpgroup: producer, two MMA issuers and an idle warp that exists
+  // only because the exchange is made by whole warpgroups) to the softmax warps, whose threads hold a row of 128
+  // scores: 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168.  Each role's branch changes its own allotment.
   if (warp == 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
     // ======================= TMA producer =======================
     if (lane == 0) {
       tma_prefetch_desc(&tm_pool);
@@ -490,6 +497,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       ok = __shfl_sync(0xffffffffu, ok, 0);
     }
   } else if (warp == 9 || warp == 10) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
     // ======================= MMA issuer =======================
     // The whole warp walks the loop converged (waits, descriptor arithmetic); one elected lane issues.
     {
@@ -580,7 +588,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       if (elect_one()) tc_commit(bar(BAR_OFINAL + i));
       __syncwarp();
     }
+  } else if (warp == 11) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX) : "memory");
     // ======================= softmax warps =======================
     // 4 warps per Q tile: TMEM lane = row = thread, which holds all 128 scores of its row in registers, so row
     // maxima and sums need no exchange.  P is written to TMEM in four quarters of 32 keys and posted to the MMA
@@ -1041,10 +1052,7 @@ constexpr int OFF_Q = 0, OFF_K = QBUF * TILE_BYTES, OFF_V = OFF_K + KV_BYTES, OF
 constexpr int SMEM = OFF_STAGE + TILE_BYTES + 1024;   // 225 KB: Q 64, K 64, V 64, output staging 32
 constexpr int SLOTS = 16;
 constexpr int THREADS = 384;  // 8 softmax warps + producer + S issuer + output store warp + PV issuer
-// Registers per thread after the roles have split (the launch gives every thread the same number; a request for
-// more blocks until other warps of the block have given theirs up, so the sum must not pass what the launch gave:
-// checked against the compiled kernel before every launch)
-constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 224;
+// (registers move between the roles as in the tile kernel: REGS_SERVICE, REGS_SOFTMAX)
 enum { B_QFULL = 0, B_QEMPTY = 2, B_SFULL = 4, B_PFULL = 6, B_OFULL = 8, B_OFREE = 10, B_STAGED = 12, B_STGFREE = 13,
        B_PHALF = 14 /* the first 64 keys of P posted */, B_DRAIN = 16 /* every MMA of a finished stream has run */,
        B_KP = 17, B_VP = 17 + SLOTS, NBARS = 17 + 2 * SLOTS };
@@ -1496,19 +1504,22 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   }
 }
 
+// The role split asks for 8 x 32 x REGS_SOFTMAX + 4 x 32 x REGS_SERVICE registers; a block that was launched with
+// fewer would wait for them for ever.
+template <typename Kernel>
+cudaError_t check_register_budget(Kernel kernel, int threads) {
+  cudaFuncAttributes attr;
+  cudaError_t e = cudaFuncGetAttributes(&attr, kernel);
+  if (e != cudaSuccess) return e;
+  return attr.numRegs * threads < 128 * REGS_SERVICE + 256 * REGS_SOFTMAX ? cudaErrorLaunchOutOfResources : cudaSuccess;
+}
+
 cudaError_t launch_stream(const CUtensorMap& tm_q, const CUtensorMap& tm_k16, const CUtensorMap& tm_v16, const CUtensorMap& tm_out,
                           int tma_out, const PrefillParams& p, int num_sms, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(prefill_swa_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, stream::SMEM);
   if (e != cudaSuccess) return e;
-  static int regs_at_launch = 0;
-  if (regs_at_launch == 0) {
-    cudaFuncAttributes attr;
-    e = cudaFuncGetAttributes(&attr, prefill_swa_stream_kernel);
-    if (e != cudaSuccess) return e;
-    regs_at_launch = attr.numRegs;
-  }
-  // the softmax warps' request for registers would never be granted
-  if (regs_at_launch * stream::THREADS < 128 * stream::REGS_SERVICE + 256 * stream::REGS_SOFTMAX) return cudaErrorLaunchOutOfResources;
+  static const cudaError_t budget = check_register_budget(prefill_swa_stream_kernel, stream::THREADS);
+  if (budget != cudaSuccess) return budget;
   const int ns_max = (p.max_q_len - 128 + stream::SUB - 1) / stream::SUB;
   if (ns_max <= 0) return cudaSuccess;
   const long long units = (long long)p.b.B * p.m.Hkv * ns_max;
@@ -1543,6 +1554,8 @@ cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap
   if (p.b.B == 0 || p.total_q == 0 || p.max_q_len == 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
+  static const cudaError_t budget = check_register_budget(prefill_tc_kernel<false>, NUM_THREADS);
+  if (budget != cudaSuccess) return budget;
   int max_tiles = (p.max_q_len + BM - 1) / BM;
   if (tile_limit > 0 && tile_limit < max_tiles) max_tiles = tile_limit;
   dim3 grid(p.m.G / 2, p.m.Hkv, (unsigned)(p.b.B * max_tiles));
@@ -1558,6 +1571,8 @@ cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensor
   if (p.b.B == 0 || n_slices <= 0) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
+  static const cudaError_t budget = check_register_budget(prefill_tc_kernel<true>, NUM_THREADS);
+  if (budget != cudaSuccess) return budget;
   dim3 grid(n_slices, p.m.Hkv, (p.b.B + 31) / 32);
   prefill_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_pool, tm_pool, p, 1);
   return cudaGetLastError();
