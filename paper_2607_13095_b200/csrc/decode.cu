@@ -176,6 +176,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
   constexpr int CHUNKS = D / 8;  // 16-byte chunks per row
   constexpr int KS = D / 16;
   static_assert(TK % P == 0, "page size must divide the tile");
+  // Consumer warp c takes tiles c, c + NW, ...: with NS a multiple of NW every fill of a stage is waited for by the
+  // same warp, so that warp sees each phase of the stage's barrier in turn.  A parity wait tells a phase only from
+  // its neighbours: a warp that skipped phases could pass a barrier that is still one fill behind.
+  static_assert(NS % NW == 0, "a stage must always be consumed by the same warp");
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * NS];
@@ -521,11 +525,19 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
   // the warp of token w patches row w into the staged tile and writes it to the cache; a barrier among the
   // token warps makes all nq rows visible before any of them reads the tiles.
   const int nq = TOKENS ? p.nq : 1;
+  // One token per request: consumer warp c takes tiles c, c + NW, ... of every ring.  When the tiles of a ring are a
+  // multiple of NW = NS (the paper's ring: 3 tiles) or a single one, a stage is always consumed by the same warp, which
+  // therefore sees each phase of the stage's barrier in turn.  Otherwise every warp waits for every tile and releases
+  // it, and works only on its own: a parity wait tells a phase only from its neighbours, so a warp that skipped
+  // phases could pass a barrier that is still one fill behind.
+  static_assert(NS == NW, "stage ownership below assumes as many stages as consumer warps");
+  const bool lockstep = !TOKENS && n_tiles != 1 && n_tiles % NW != 0;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(smem_u32(&bars[i]), 1);
-      mbar_init(smem_u32(&bars[NS + i]), TOKENS ? nq : 1);  // consumers that release a tile: one per token, or its one warp
+      // consumers that release a tile: one per token; else the one warp that works on it, or all of them in lockstep
+      mbar_init(smem_u32(&bars[NS + i]), TOKENS ? nq : (lockstep ? NW : 1));
     }
     mbar_fence_init();
     tma_prefetch_desc(&tm_pool);
@@ -804,12 +816,16 @@ decode_ring_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodePara
 #pragma unroll
       for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
       bool ok = true;
-      for (int t = cw; t < n_tiles; t += NW) {
+      for (int t = lockstep ? 0 : cw; t < n_tiles; t += lockstep ? 1 : NW) {
         const int g = k * n_tiles + t, stage = g % NS;
         if (!mbar_wait(smem_u32(&bars[stage]), (g / NS) & 1)) {
           if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, t, 4);
           ok = false;
           break;
+        }
+        if (lockstep && t % NW != cw) {
+          if (lane == 0) mbar_arrive(smem_u32(&bars[NS + stage]));
+          continue;
         }
         uint8_t* sK = smem + stage * STAGE_BYTES;
         uint8_t* sV = sK + HALVES * HALF_BYTES;
@@ -936,7 +952,7 @@ struct KeyRangeMulti {
 };
 
 template <int D, int P, int NS>
-__global__ void __launch_bounds__(160, 2)
+__global__ void __launch_bounds__(160, 3)
 decode_mtp_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p) {
   constexpr int HALVES = D / 64;
   constexpr int PPT = TK / P;
@@ -1171,9 +1187,9 @@ cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool,
   if (D == 128 && P == 64) return launch_decode_t<128, 64, 3, 3>(tm_pool, p, early_start, s);
   if (D == 128 && P == 32) return launch_decode_t<128, 32, 3, 3>(tm_pool, p, early_start, s);
   if (D == 128 && P == 16) return launch_decode_t<128, 16, 3, 3>(tm_pool, p, early_start, s);
-  if (D == 64 && P == 64) return launch_decode_t<64, 64, 4, 3>(tm_pool, p, early_start, s);
-  if (D == 64 && P == 32) return launch_decode_t<64, 32, 4, 3>(tm_pool, p, early_start, s);
-  if (D == 64 && P == 16) return launch_decode_t<64, 16, 4, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 64) return launch_decode_t<64, 64, 3, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 32) return launch_decode_t<64, 32, 3, 3>(tm_pool, p, early_start, s);
+  if (D == 64 && P == 16) return launch_decode_t<64, 16, 3, 3>(tm_pool, p, early_start, s);
   return cudaErrorInvalidValue;
 }
 
@@ -1200,9 +1216,9 @@ cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_p
   if (p.nq < 1 || p.nq > 4) return cudaErrorInvalidValue;
   if (p.is_swa) return hswa_launch_decode(h, tm_pool, p, early_start, s);  // rings: one work item per (ring, token)
   const int D = p.m.D, P = p.m.P;
-  if (D == 128 && P == 64) return launch_mtp_t<128, 64, 3>(tm_pool, p, s);
-  if (D == 128 && P == 32) return launch_mtp_t<128, 32, 3>(tm_pool, p, s);
-  if (D == 128 && P == 16) return launch_mtp_t<128, 16, 3>(tm_pool, p, s);
+  if (D == 128 && P == 64) return launch_mtp_t<128, 64, 2>(tm_pool, p, s);
+  if (D == 128 && P == 32) return launch_mtp_t<128, 32, 2>(tm_pool, p, s);
+  if (D == 128 && P == 16) return launch_mtp_t<128, 16, 2>(tm_pool, p, s);
   if (D == 64 && P == 64) return launch_mtp_t<64, 64, 4>(tm_pool, p, s);
   if (D == 64 && P == 32) return launch_mtp_t<64, 32, 4>(tm_pool, p, s);
   if (D == 64 && P == 16) return launch_mtp_t<64, 16, 4>(tm_pool, p, s);

@@ -1053,9 +1053,9 @@ constexpr int SMEM = OFF_STAGE + TILE_BYTES + 1024;   // 225 KB: Q 64, K 64, V 6
 constexpr int SLOTS = 16;
 constexpr int THREADS = 384;  // 8 softmax warps + producer + S issuer + output store warp + PV issuer
 // (registers move between the roles as in the tile kernel: REGS_SERVICE, REGS_SOFTMAX)
-enum { B_QFULL = 0, B_QEMPTY = 2, B_SFULL = 4, B_PFULL = 6, B_OFULL = 8, B_OFREE = 10, B_STAGED = 12, B_STGFREE = 13,
-       B_PHALF = 14 /* the first 64 keys of P posted */, B_DRAIN = 16 /* every MMA of a finished stream has run */,
-       B_KP = 17, B_VP = 17 + SLOTS, NBARS = 17 + 2 * SLOTS };
+enum { B_QFULL = 0, B_QEMPTY = 2, B_SFULL = 4, B_PFULL = 6, B_OFULL = 8, B_OFREE = 10, B_STAGED = 12,
+       B_PHALF = 13 /* the first 64 keys of P posted */, B_DRAIN = 15 /* every MMA of a finished stream has run */,
+       B_STGFREE = 16 /* two: staged tiles use them in turn */, B_KP = 18, B_VP = 18 + SLOTS, NBARS = 18 + 2 * SLOTS };
 // instruction descriptor of an S MMA over n keys (a multiple of 16)
 __device__ __forceinline__ uint32_t idesc_s(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -1139,6 +1139,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   if (threadIdx.x == 0) {
     mbar_init(bar(B_STAGED), 4);
     mbar_init(bar(B_STGFREE), 1);
+    mbar_init(bar(B_STGFREE + 1), 1);
     mbar_init(bar(B_DRAIN), 1);
     for (int q = 0; q < QBUF; ++q) {
       mbar_init(bar(B_QFULL + q), 1);
@@ -1341,7 +1342,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                        : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory has been read
-        mbar_arrive(bar(B_STGFREE));
+        mbar_arrive(bar(B_STGFREE + (n_staged & 1)));
         ++n_staged;
       }
       if (!ok) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, n_staged, 73);
@@ -1459,7 +1460,14 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
           // (the row is scaled and packed first: that work needs no staging tile)
 #pragma unroll
           for (int c = 0; c < 64; ++c) wv[c] = pack_bf16x2(__uint_as_float(wv[2 * c]) * inv, __uint_as_float(wv[2 * c + 1]) * inv);
-          if (my_stage_idx > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(B_STGFREE), (my_stage_idx - 1) & 1))) {
+          // Staged tile k waits until the store of tile k - 1 has read the staging tile.  The two warpgroups mostly
+          // alternate, so this warpgroup saw the barrier of tile k - 2 at best: with ONE barrier it would wait for
+          // a phase without having seen the one before, and a parity wait passes at once when the barrier is a
+          // whole phase behind (a late store warp: corrupted tiles, miscounted arrivals).  With two barriers used
+          // in turn, the phase before the awaited one belongs to tile k - 3, whose store this warpgroup's own
+          // earlier wait (for k - 3 or k - 2) has already covered.
+          if (my_stage_idx > 0 &&
+              !__all_sync(0xffffffffu, mbar_wait(bar(B_STGFREE + ((my_stage_idx - 1) & 1)), ((my_stage_idx - 1) >> 1) & 1))) {
             if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, g, 75);
           }
 #pragma unroll

@@ -47,7 +47,7 @@ def test_block_orders_agree_and_longest_first_is_descending_work():
         out = torch.full((t.total_q, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
         traces.append(run_with_trace(h, layer, b, q, k, v, out, blocks))
         outs.append(out.cpu().numpy())
-        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
     assert np.abs(outs[0] - ref).max() <= TOL
     assert all(np.array_equal(outs[0], o) for o in outs[1:])   # the order changes no bit
@@ -106,7 +106,7 @@ def test_longest_first_shrinks_the_idle_tail_of_a_mixed_length_batch():
         last_on_sm = np.array([tr[tr[:, 2] == s, 1].max() for s in np.unique(tr[:, 2])])
         idle[mode] = float((end - last_on_sm).mean() / (end - start))   # mean idle tail of an SM, as a share of the span
         outs[mode] = out.view(torch.int16).cpu().numpy()
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     for mode in (hb.PREFILL_ORDER_LONGEST_REQUEST_FIRST, hb.PREFILL_ORDER_LONGEST_TILE_FIRST):
         assert np.array_equal(outs[hb.PREFILL_ORDER_BY_REQUEST], outs[mode])
         assert idle[mode] < idle[hb.PREFILL_ORDER_BY_REQUEST], idle
@@ -145,7 +145,8 @@ def test_chunked_prefill_at_the_longest_prefixes(prefix):
         out = torch.zeros((chunk, d.num_q_heads, d.head_dim), dtype=torch.bfloat16, device="cuda")
         hb.hswa_prefill_attn(h, hb.Layer(pool, is_swa), b, q, k, v, True, out, None, None)
         torch.cuda.synchronize()
-        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+        async_err = hb.hswa_get_async_error(h)
+        assert async_err[0] == hb.HSWA_OK, (is_swa, async_err)
         tok = np.array(special + list(rng.integers(0, chunk, n_rows - len(special))), dtype=np.int32)
         head = rng.integers(0, d.num_q_heads, len(tok)).astype(np.int32)
         layer = orc.OracleLayer(before, is_swa)

@@ -56,7 +56,7 @@ def test_exact_workspace_need_is_the_acceptance_threshold():
         hb.hswa_decode_attn(h, layer, dev_batch(t, True), q, k, v, out, None, ws[: need - 256])
     assert e.value.status == hb.HSWA_ERR_WORKSPACE
     hb.hswa_decode_attn(h, layer, dev_batch(t, True), q, k, v, out, None, ws)
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
     assert np.abs(out.cpu().numpy() - ref).max() <= TOL
 
@@ -78,7 +78,7 @@ def test_mtp_rejects_windows_too_long_for_either_ring_kernel_without_launching()
     with pytest.raises(hb.HswaError) as e:
         hb.hswa_decode_attn_mtp(h, swa, b, 2, q, k, v, out, None, workspace_for(h, t))
     assert e.value.status == hb.HSWA_ERR_UNSUPPORTED
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     assert (out == 7.0).all() and np.array_equal(to_host_bits(swa.pool), before)   # nothing ran
 
 
@@ -110,7 +110,7 @@ def test_ring_decode_other_windows_and_token_counts(W, P, D, G, nq):
         hb.hswa_decode_attn(h, layer, b, q, k, v, out, lse, None)
     else:
         hb.hswa_decode_attn_mtp(h, layer, b, nq, q, k, v, out, lse, None)
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     ol = sc.layer(True)
     ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
     got = out.cpu().numpy().astype(np.float64)
@@ -129,7 +129,7 @@ def test_single_token_decode_serves_long_rings():
     out = torch.zeros((t.batch, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
     hb.hswa_decode_attn(h, swa, dev_batch(t, True), to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new), out,
                         None, workspace_for(h, t))
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     ol = sc.layer(True)
     ref, _ = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
     assert np.abs(out.cpu().numpy() - ref).max() <= TOL
@@ -165,7 +165,7 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     st = hb.hswa_get_async_error(h)
     assert st == (hb.HSWA_ERR_TIMEOUT, -1, 0, 7), st
     assert t0.elapsed_time(t1) < 1000.0            # it did give up at the limit
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     with pytest.raises(hb.HswaError):
         hb.hswa_selftest_wait_timeout(h, 0)
     # the library still works on this context
@@ -175,7 +175,7 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     out = torch.zeros((t.batch, d.num_q_heads, d.head_dim), dtype=torch.float32, device="cuda")
     hb.hswa_decode_attn(h, layer, dev_batch(t, True), to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new), out,
                         None, workspace_for(h, t))
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     ref, _ = orc.attention(sc.cfg, sc.layer(False), sc.batch(), sc.q, sc.k_new, sc.v_new)
     assert np.abs(out.cpu().numpy() - ref).max() <= TOL
 
@@ -207,7 +207,7 @@ def test_early_start_chain_next_to_foreign_kernels(is_swa):
         hb.hswa_decode_attn(h, layers[i], b, q, k, v, outs[i], None, ws)
     # same layer again, right behind its own fused decode, reading the row that call appended
     hb.hswa_decode_attn(h, layers[2], b, q, None, None, outs[3], None, ws)
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     for i in range(3):
         scaled = [to_host_bits((x * scales[i]).contiguous()) for x in (q_src, k_src, v_src)]
         ol = sc.layer(is_swa)
@@ -237,7 +237,7 @@ def test_overlap_switched_off_allows_foreign_pool_writes():
         hb.hswa_decode_attn(h, first, b, q, k, v, outs[0], None, ws)
         second.pool.copy_(src)                              # foreign kernel writes the next layer's pool
         hb.hswa_decode_attn(h, second, b, q, k, v, outs[1], None, ws)
-        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
         ol = sc.layer(is_swa)
         ref, _ = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
         orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)

@@ -318,7 +318,7 @@ def test_validate_batch_reports_bad_ids():
     swa = hb.Layer(to_dev_bf16(sc.swa_pool), True)
     hb.hswa_validate_batch(h, full, dev_batch(t, True))
     hb.hswa_validate_batch(h, swa, dev_batch(t, True))
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     # corrupt the HOST copy of the block table, then validate: the error word names request and entry
     bad = t.block_table.copy()
     bad[1, 0] = t.num_full_pages + 7
@@ -393,7 +393,7 @@ def test_host_side_argument_errors():
     empty = hb.Batch(dev_i32(np.zeros(0)), dev_i32(np.zeros((0, 1))), dev_i32(np.zeros((0, 3))), dev_i32(np.zeros(0)),
                      max_q_len=1, total_q=0)
     hb.hswa_decode_attn(h, full, empty, q, None, None, out, None, None)
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
 
 
 # ---------------------------------------------------------------------------------------------------------

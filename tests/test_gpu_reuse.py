@@ -84,7 +84,7 @@ def test_release_then_window_safe_hit_then_seeded_decode(d, every_n):
         hb.hswa_swa_release(h, B, ctx, torch.from_numpy(flags).cuda(), valid_from)
         orc.swa_release(cfg, octx, flags, ofrom)
         assert np.array_equal(valid_from.cpu().numpy(), ofrom), (kind, who, arg)
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     assert octx.tolist() == total
     for s in (False, True):
         assert np.array_equal(to_host_bits(pools[s]), o_pools[s])
@@ -171,7 +171,7 @@ def test_release_then_window_safe_hit_then_seeded_decode(d, every_n):
     hb.hswa_step_advance(h, 1, nb.ctx_len, nb.ring_head, None)
     hb.hswa_swa_release(h, 1, nb.ctx_len, None, new_from)
     assert new_from.cpu().numpy().tolist() == [max(0, L + 1 - (W - 1))]
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
 
 
 def test_layerwise_loadback_equals_resident_run():
@@ -229,7 +229,7 @@ def test_layerwise_loadback_equals_resident_run():
         main.wait_event(events[i])
         hb.hswa_decode_attn(h, hb.Layer(reloaded[i], True), b, q[i], k[i], v[i], out[i], None, None)
     torch.cuda.synchronize()
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
     assert torch.equal(out.view(torch.int16), want.view(torch.int16))   # same bits as the resident run
     # and right: the oracle on the resident rings (one layer)
     cfg = oracle_config(d)

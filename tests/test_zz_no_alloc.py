@@ -31,7 +31,7 @@ def _both(sc, is_swa):
             hb.hswa_decode_attn_static_ws(h, layer, dev_batch(t, True), q, k, v, out, lse)
         else:
             hb.hswa_decode_attn(h, layer, dev_batch(t, True), q, k, v, out, lse, workspace_for(h, t))
-        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+        assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
         res.append((out.cpu().numpy(), lse.cpu().numpy(), layer.pool.view(torch.int16).cpu().numpy()))
     (o0, l0, p0), (o1, l1, p1) = res
     assert np.isfinite(o1).all()
@@ -71,4 +71,4 @@ def test_static_ws_rejects_oversized_batch():
     with pytest.raises(hb.HswaError) as e:
         hb.hswa_decode_attn_static_ws(h, layer, big, to_dev_bf16(sc.q), None, None, out)
     assert e.value.status == hb.HSWA_ERR_WORKSPACE
-    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK
+    assert hb.hswa_get_async_error(h)[0] == hb.HSWA_OK, hb.hswa_get_async_error(h)
