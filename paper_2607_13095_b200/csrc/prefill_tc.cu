@@ -312,6 +312,14 @@ __device__ __forceinline__ long long global_timer_ns() {
   return t;
 }
 
+// Called by every thread on its way out.  A role that gave up (a wait ran out, an error was recorded) leaves its
+// loop while TMA loads that nobody will wait for may still be in flight towards this block's shared memory; a block
+// must not exit, and hand its shared memory to the next block, before they have landed.  No barrier says when that
+// is once the protocol is broken, so the error path simply outwaits them (0.1 ms, far above any TMA latency).
+__device__ __forceinline__ void linger_after_error(const int32_t* err) {
+  if (*reinterpret_cast<const volatile int32_t*>(err) != 0) __nanosleep(100000);
+}
+
 // PREFIX = true turns the same pipeline into the shared-prefix stage of batched decode (paper Sec. 3.1.3 /
 // 3.1.4: requests that share a system prompt share its pages): the 128 rows of a Q tile are 16 requests x
 // the 8 query heads of one KV head, the keys are a slice of the shared prefix pages, nothing is masked, and
@@ -806,6 +814,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   }
 
   // ---- teardown: everyone is done with TMEM before it is released ----
+  linger_after_error(p.err);
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
@@ -1504,6 +1513,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
       }
     }
   }
+  linger_after_error(p.err);
   tc_fence_before();
   __syncthreads();
   if (warp == 8) {
