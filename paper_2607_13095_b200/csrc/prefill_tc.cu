@@ -1135,6 +1135,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   // what the softmax warps need to know about a sub-tile, written by the producer when it issues the Q load:
   // {first token (row of q / out), valid tokens, KV head, index among the staged tiles or -1}
   __shared__ int4 tile_info[4];
+  __shared__ int blk_abort;  // a wait of a softmax warp ran out: both warpgroups stop at their next sub-tile
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
@@ -1146,6 +1147,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 
   auto bar = [&](int i) { return smem_u32(&bars[i]); };
   if (threadIdx.x == 0) {
+    blk_abort = 0;
     mbar_init(bar(B_STAGED), 4);
     mbar_init(bar(B_STGFREE), 1);
     mbar_init(bar(B_STGFREE + 1), 1);
@@ -1367,7 +1369,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint32_t tS = tmem + lane_addr + u * 256, tO = tS + 128;
     const int lo = tl + 129 - M.W, hi = tl + 129;  // visible key columns [lo, hi) of the 144-key slice
     const int n_total = count_sub_tiles(p, ns_max, u0, u1);
-    for (int g = u; g < n_total; g += 2) {
+    for (int g = u; g < n_total && *reinterpret_cast<volatile int*>(&blk_abort) == 0; g += 2) {
       const uint32_t par = (g >> 1) & 1;
       bool ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SFULL + u), par));
       float l_run = 0.f, m_use = 0.f;
@@ -1434,6 +1436,7 @@ prefill_swa_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         if (lane == 0) {
           record_error(p.err, HSWA_ERR_TIMEOUT, blockIdx.x, g, 74);
           mbar_arrive(bar(B_PHALF + u));
+          *reinterpret_cast<volatile int*>(&blk_abort) = 1;
         }
       }
       tc_fence_before();
