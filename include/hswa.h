@@ -47,6 +47,10 @@
  *   keys j in [lo, p], lo = 0 on a Full layer and max(0, p - W + 1) on an SWA layer (W keys including the
  *   query's own position); out = softmax(sm_scale * q K^T) V with fp32 accumulation, lse = natural-log
  *   log-sum-exp of the scaled scores.
+ *   Slots that hold no key of [lo, p] (page tails behind the cached context, ring slots older than the window or
+ *   never written, pages no request refers to) may contain anything, bit patterns of NaN and infinity included:
+ *   no decode or prefill call lets them change a result (Sec. 3.1.3: attention must not read invalid or
+ *   overwritten slots).
  *
  * Supported shapes: D in {64, 128}; P in {16, 32, 64}; 1 <= G <= 8; W >= 1; R * P >= W + 1.
  */

@@ -34,7 +34,7 @@ constexpr int PG = 64;                // page size
 constexpr int HALF_BYTES = 128 * 128; // [128 rows][128 B]: one 64-element half of a 128-row tile
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 constexpr int KV_STAGES = 2;
-constexpr int NUM_THREADS = 384;  // 8 softmax warps + producer + one MMA issuer per Q tile + an idle warp (see the kernel)
+constexpr int NUM_THREADS = 384;  // 8 softmax warps + producer + one MMA issuer per Q tile + the patch warp
 // Registers per thread after the roles have split; the sum over the block must not pass what the launch gave
 // (384 x 168), or the softmax warps' request would never be granted: checked against the compiled kernel before launch.
 constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 224;
@@ -51,7 +51,8 @@ constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [ke
 
 // barrier indices
 enum { BAR_Q = 0, BAR_KFULL = 1, BAR_KEMPTY = 3, BAR_VFULL = 5, BAR_VEMPTY = 7, BAR_SFULL = 9,
-       BAR_PFULL = 11 /* [Q tile][half of the key columns] */, BAR_OFINAL = 15 /* [Q tile] */, NUM_BARS = 17 };
+       BAR_PFULL = 11 /* [Q tile][half of the key columns] */, BAR_OFINAL = 15 /* [Q tile] */,
+       BAR_VPATCH = 17 /* [stage]: a V tile whose dead rows are zeroed before the MMA issuers see it */, NUM_BARS = 19 };
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -324,6 +325,11 @@ __device__ __forceinline__ void linger_after_error(const int32_t* err) {
 // 3.1.4: requests that share a system prompt share its pages): the 128 rows of a Q tile are 16 requests x
 // the 8 query heads of one KV head, the keys are a slice of the shared prefix pages, nothing is masked, and
 // the block writes an unnormalised (m, l, o) partial per row for the split-K combine instead of an output.
+// Does cached tile j (of nA) of a request with ctx cached tokens hold rows that no row of the block can see?  On a
+// Full layer: the last tile when ctx ends inside it.  On an SWA layer: every ring tile (slots older than the window,
+// never written, or past the ring's last page).
+__device__ __forceinline__ bool v_tile_needs_patch(int is_swa, int ctx, int j) { return is_swa || ctx - j * BN < BN; }
+
 template <bool PREFIX>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_constant__ CUtensorMap tm_q,
@@ -421,6 +427,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
     mbar_init(bar(BAR_OFINAL), 1);
     mbar_init(bar(BAR_OFINAL + 1), 1);
+    static_assert(KV_STAGES == 2, "one patch barrier per V stage");
+    mbar_init(bar(BAR_VPATCH), 1);
+    mbar_init(bar(BAR_VPATCH + 1), 1);
     mbar_fence_init();
   }
   if (warp == 8) {
@@ -433,9 +442,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   tc_fence_after();
   const uint32_t tmem = tmem_base_slot;
 
-  // Registers move from the service warps (one warpgroup: producer, two MMA issuers and an idle warp that exists
-  // only because the exchange is made by whole warpgroups) to the softmax warps, whose threads hold a row of 128
-  // scores: 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168.  Each role's branch changes its own allotment.
+  // Registers move from the service warps (one warpgroup: producer, two MMA issuers and the patch warp; the
+  // exchange is made by whole warpgroups) to the softmax warps, whose threads hold a row of 128 scores:
+  // 8 x 32 x 224 + 4 x 32 x 56 = 384 x 168.  Each role's branch changes its own allotment.
   if (warp == 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
     // ======================= TMA producer =======================
@@ -462,6 +471,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     for (int j = 0; j < n_tiles && ok; ++j) {
       const int stage = j % KV_STAGES;
       int pg[2] = {0, 0};
+      // Rows of a cached tile that no row of this block can see (the tail of the last page of a Full layer; ring
+      // slots never written, past the ring's last page, or older than the first row's window, which a ring seeded
+      // with a window only never filled) may hold anything, patterns of NaN included.  Their probabilities are exactly
+      // 0, but 0 x NaN would still reach the output through the PV MMA (paper Sec. 3.1.3: attention must not be
+      // affected by invalid slots).  The V half of such a tile lands on a barrier that the patch warp (warp 11)
+      // waits on; that warp zeroes the dead rows and only then hands the tile to the MMA issuers.
+      const bool patch = !PREFIX && j < seq.nA && v_tile_needs_patch(p.is_swa, ctx, j);
       if (j < seq.nA) {
         if (((2 * j) & 31) == 0) {
           pid_cur = pid_next;
@@ -478,12 +494,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
         const uint32_t par = ((j / KV_STAGES) - 1) & 1;
         const uint32_t dK = sbase + OFF_K + stage * TILE_BYTES, dV = sbase + OFF_V + stage * TILE_BYTES;
         for (int kv = 0; kv < 2 && ok; ++kv) {
-          const uint32_t full = bar((kv ? BAR_VFULL : BAR_KFULL) + stage);
+          const uint32_t full_mma = bar((kv ? BAR_VFULL : BAR_KFULL) + stage);
           if (j >= KV_STAGES && !mbar_wait(bar((kv ? BAR_VEMPTY : BAR_KEMPTY) + stage), par)) {
             record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 10 + kv);
             ok = false;
             break;
           }
+          const uint32_t full = (kv && patch) ? bar(BAR_VPATCH + stage) : full_mma;
           mbar_arrive_expect_tx(full, TILE_BYTES);
           const uint32_t dst = kv ? dV : dK;
           if (j < seq.nA) {
@@ -598,6 +615,40 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
   } else if (warp == 11) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_SERVICE) : "memory");
+    // ======================= patch warp =======================
+    // (see the producer: dead rows of a cached V tile are zeroed between the tile's arrival and its hand-over)
+    if constexpr (!PREFIX) {
+      uint32_t n_patched = 0;  // bit s: parity of the next patch of stage s
+      for (int j = 0; j < seq.nA; ++j) {
+        if (!v_tile_needs_patch(p.is_swa, ctx, j)) continue;
+        const int stage = j % KV_STAGES;
+        // the producer arms this barrier once per patched tile of the stage, after the stage's previous tile has been
+        // consumed: this warp sees each of its phases in turn
+        if (!mbar_wait(bar(BAR_VPATCH + stage), (n_patched >> stage) & 1u)) {
+          if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 12);
+          break;
+        }
+        n_patched ^= 1u << stage;
+        uint8_t* sV = smem + OFF_V + stage * TILE_BYTES;
+        for (int idx = lane; idx < BN * 16; idx += 32) {  // 16-byte chunks: 128 rows x 2 halves x 8
+          const int row = (idx >> 3) & (BN - 1), hf = idx >> 10, ch = idx & 7;
+          bool live;
+          if (!p.is_swa) {
+            live = row < ctx - j * BN;
+          } else {
+            const int slot = j * BN + row;  // ring slot; it holds position kpos = ctx - C + ((slot - head) mod C)
+            int off = slot - head;
+            if (off < 0) off += M.C;
+            const int kpos = ctx - M.C + off;
+            live = slot < M.C && kpos >= 0 && kpos > ctx + b * BM - M.W;  // visible to the block's first row at least
+          }
+          if (!live) *reinterpret_cast<uint4*>(sV + hf * HALF_BYTES + row * 128 + ch * 16) = make_uint4(0, 0, 0, 0);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(BAR_VFULL + stage));
+      }
+    }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX) : "memory");
     // ======================= softmax warps =======================

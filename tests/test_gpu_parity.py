@@ -454,6 +454,28 @@ def test_prefill_tc_long_context_and_many_requests():
         assert err <= TOL and lerr <= TOL, (is_swa, err, lerr)
 
 
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(2, 128, 64, 3), dims(4, 64, 16, 1)], ids=str)
+@pytest.mark.parametrize("is_swa", [False, True])
+def test_prefill_ignores_nonfinite_dead_slots(d, is_swa):
+    """As test_decode_ignores_nonfinite_stale_slots, for chunked prefill: slots that hold no token (page tails behind
+    the cached context, ring slots never written or past the ring's last page, unused pages) hold +inf (K) and NaN
+    (V).  Their probabilities are exactly 0, and 0 * NaN must not reach the output through the PV product either
+    (Sec. 3.1.3).  Contexts that end inside a 128-key tile, inside a page, and rings that are not full yet."""
+    from helpers import POISON_K, POISON_V
+    W, C = d.window, d.ring_slots
+    ctx = [0, 1, 5, 63, 64, 65, 100, W - 1, W, W + 1, C - 1, C, C + 7, 1000, 2049]
+    q_len = [130, 64, 300, 129, 1, 128, 257, 70, 200, 16, 140, 131, 5, 260, 129]
+    sc = build_scenario(d, ctx, q_len, seed=92)
+    pk, pv = wl.bf16_bits_const(POISON_K, (1,))[0], wl.bf16_bits_const(POISON_V, (1,))[0]
+    for pool in (sc.full_pool, sc.swa_pool):
+        assert int((pool[:, 0] == pk).sum()) > 0 and int((pool[:, 1] == pv).sum()) > 0
+        pool[:, 0][pool[:, 0] == pk] = 0x7F80  # +inf
+        pool[:, 1][pool[:, 1] == pv] = 0x7FC0  # NaN
+    for fuse_append in (True, False):
+        err, lerr = run_prefill(sc, is_swa, fuse_append)
+        assert err <= TOL and lerr <= TOL, (fuse_append, err, lerr)
+
+
 @pytest.mark.parametrize("case", ["many_short_streams", "one_long_stream", "two_long_streams", "fewer_units_than_sms"])
 def test_prefill_swa_stream_walk(case):
     """The streaming SWA kernel (group of 8, W = 128) hands each persistent block a run of 16-token sub-tiles that may
