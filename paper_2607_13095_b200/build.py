@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhswa.so")
-SOURCES = ["api.cu", "cache_ops.cu", "decode.cu", "decode_ring.cu", "decode_static_ws.cu", "prefill_mma.cu", "prefill_tc.cu"]
+SOURCES = ["api.cu", "cache_ops.cu", "decode.cu", "decode_ring.cu", "decode_static_ws.cu", "decode_mtp_tc.cu", "prefill_mma.cu", "prefill_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

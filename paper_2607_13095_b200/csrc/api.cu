@@ -82,6 +82,8 @@ struct DecodePlan {
   int k_start, split_base;        // first key and first partial slot of the streaming kernel
   int split_len, grid_splits, max_splits;
   size_t o_bytes, ml_bytes;       // scratch: o partials, then (m, l) pairs; 0 when rows are written directly
+  bool tc;                        // multi-token decode on the tensor cores: run partials and one int2 per stream
+  size_t info_bytes;
 };
 
 bool plan_decode(const hswa_handle* h, int is_swa, int batch, int max_ctx_len, int shared_prefix_len, int q_len,
@@ -89,9 +91,15 @@ bool plan_decode(const hswa_handle* h, int is_swa, int batch, int max_ctx_len, i
   DecodePlan d = {};
   d.cascade = !is_swa && q_len == 1 && shared_prefix_len >= 128 && h->cfg.head_dim == 128 && h->cfg.page_size == 64 &&
               h->group == 8;
+  d.tc = !is_swa && q_len >= 2 && hswa_decode_mtp_tc_supported(model_params(h), batch, q_len);
   if (is_swa) {
     d.split_len = ((h->ring_slots + 63) / 64) * 64;
     d.grid_splits = d.max_splits = 1;
+  } else if (d.tc) {
+    d.split_len = 128;
+    d.grid_splits = 1;
+    d.max_splits = 2;
+    hswa_decode_mtp_tc_scratch(model_params(h), batch, h->num_sms, &d.o_bytes, &d.ml_bytes, &d.info_bytes);
   } else {
     if (d.cascade) {
       const int tiles = (shared_prefix_len + 127) / 128;
@@ -249,7 +257,12 @@ size_t hswa_workspace_bytes(const hswa_handle* h, int32_t max_batch, int32_t max
                             (size_t)32 * h->group * h->num_sms;
   const size_t o_bytes = row_splits * h->cfg.head_dim * sizeof(float);
   const size_t ml_bytes = row_splits * sizeof(float2);
-  return ((o_bytes + 255) & ~size_t(255)) + ((ml_bytes + 255) & ~size_t(255));
+  size_t need = ((o_bytes + 255) & ~size_t(255)) + ((ml_bytes + 255) & ~size_t(255));
+  // the tensor-core multi-token path keeps partials per run (streams + blocks of them), not per row and split
+  size_t tc_o, tc_ml, tc_info;
+  hswa_decode_mtp_tc_scratch(model_params(h), max_batch, h->num_sms, &tc_o, &tc_ml, &tc_info);
+  if (need < tc_o + tc_ml + tc_info) need = tc_o + tc_ml + tc_info;
+  return need;
 }
 
 size_t hswa_decode_workspace_need(const hswa_handle* h, int32_t is_swa, int32_t batch, int32_t max_ctx_len,
@@ -258,7 +271,7 @@ size_t hswa_decode_workspace_need(const hswa_handle* h, int32_t is_swa, int32_t 
     return 0;
   DecodePlan pl;
   if (!plan_decode(h, is_swa, batch, max_ctx_len, shared_prefix_len, q_len, &pl)) return 0;
-  return pl.o_bytes + pl.ml_bytes;
+  return pl.o_bytes + pl.ml_bytes + pl.info_bytes;
 }
 
 hswa_status hswa_set_overlap(hswa_handle* h, int32_t enabled) {
@@ -486,7 +499,8 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   p.grid_splits = pl.grid_splits;
   p.max_splits = pl.max_splits;
   if (p.max_splits > 1) {
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 || workspace_bytes < pl.o_bytes + pl.ml_bytes)
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0 ||
+        workspace_bytes < pl.o_bytes + pl.ml_bytes + pl.info_bytes)
       return HSWA_ERR_WORKSPACE;
     p.part_o = static_cast<float*>(workspace);
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(workspace) + pl.o_bytes);
@@ -495,8 +509,15 @@ hswa_status hswa_decode_attn_mtp(hswa_handle* h, const hswa_layer* layer, const 
   const int granule = h->cfg.page_size < HSWA_RING_GRANULE ? h->cfg.page_size : HSWA_RING_GRANULE;
   if ((st = make_pool_map(h, layer, &tm, layer->is_swa ? granule : 0)) != HSWA_OK) return st;
   if (!layer->is_swa && hswa_launch_append(a, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
-  if (hswa_launch_decode_mtp(h, tm, p, early, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
-  if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  if (pl.tc) {
+    // tensor-core path: the rows of a request (tokens x heads) share one pass over its KV bytes
+    CUtensorMap tm_q;
+    if ((st = make_rows_map(h, q, h->cfg.num_q_heads, (int64_t)b->batch * q_len, 4, &tm_q, 8)) != HSWA_OK) return st;
+    if (hswa_launch_decode_mtp_tc(tm, tm_q, p, h->num_sms, workspace, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  } else {
+    if (hswa_launch_decode_mtp(h, tm, p, early, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+    if (p.max_splits > 1 && hswa_launch_combine(p, (cudaStream_t)stream) != cudaSuccess) return HSWA_ERR_CUDA;
+  }
   h->chain_ok = 1;  // none of these kernels writes the batch arrays or another layer's pool
   h->chain_stream = stream;
   h->chain_ctx = (const void*)b->ctx_len;

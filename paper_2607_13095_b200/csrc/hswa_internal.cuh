@@ -128,6 +128,11 @@ cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensor
                                             bool early_start, cudaStream_t s);
 cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
                                    bool early_start, cudaStream_t s);
+// Multi-token decode on Full layers on the tensor cores (group of 8, head_dim 128, page 64, 2-4 tokens per request)
+bool hswa_decode_mtp_tc_supported(const ModelParams& m, int batch, int nq);
+void hswa_decode_mtp_tc_scratch(const ModelParams& m, int batch, int num_sms, size_t* o_bytes, size_t* ml_bytes, size_t* info_bytes);
+cudaError_t hswa_launch_decode_mtp_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const DecodeParams& p, int num_sms,
+                                      void* scratch, cudaStream_t s);
 cudaError_t hswa_launch_prefill_mma(const PrefillParams& p, cudaStream_t s);
 bool hswa_prefill_tc_supported(const ModelParams& m);
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,

@@ -102,16 +102,10 @@ def test_decode_ignores_nonfinite_stale_slots(d, is_swa):
     """Slots that hold no valid token (stale ring slots, page tails, unused pages) are filled with +inf (K) and
     NaN (V) instead of the finite poison: decode must neither read them into a score that counts nor let
     0 * NaN reach the output (Sec. 3.1.3: reading an invalid slot degrades correctness)."""
-    from helpers import POISON_K, POISON_V
     W, C = d.window, d.ring_slots
     ctx = [0, 1, 5, 63, 64, 100, W - 1, W, W + 1, C, C + 7, 1000, 2049]
     sc = build_scenario(d, ctx, [1] * len(ctx), seed=91)
-    pk, pv = wl.bf16_bits_const(POISON_K, (1,))[0], wl.bf16_bits_const(POISON_V, (1,))[0]
-    for pool in (sc.full_pool, sc.swa_pool):
-        n_k, n_v = int((pool[:, 0] == pk).sum()), int((pool[:, 1] == pv).sum())
-        assert n_k > 0 and n_v > 0
-        pool[:, 0][pool[:, 0] == pk] = 0x7F80  # +inf
-        pool[:, 1][pool[:, 1] == pv] = 0x7FC0  # NaN
+    poison_dead_slots_nonfinite(sc)
     for fused in (True, False):
         err, lerr = run_decode(sc, is_swa, fused)
         assert err <= TOL and lerr <= TOL, (fused, err, lerr)
@@ -170,6 +164,20 @@ def test_decode_page_permutation_bit_identical():
 
 
 # ---------------------------------------------------------------------------------------------------------
+def poison_dead_slots_nonfinite(sc):
+    """Every slot of both pools that holds no token (its whole row still carries the finite poison the scenario was
+    built with) gets +inf in K and NaN in V.  Whole rows only: a valid row may contain an element whose bits happen
+    to equal the poison's."""
+    from helpers import POISON_K, POISON_V
+    pk, pv = wl.bf16_bits_const(POISON_K, (1,))[0], wl.bf16_bits_const(POISON_V, (1,))[0]
+    for pool in (sc.full_pool, sc.swa_pool):
+        dead_k = (pool[:, 0] == pk).all(axis=-1)
+        dead_v = (pool[:, 1] == pv).all(axis=-1)
+        assert dead_k.any() and dead_v.any()
+        pool[:, 0][dead_k] = 0x7F80  # +inf
+        pool[:, 1][dead_v] = 0x7FC0  # NaN
+
+
 def run_prefill(sc, is_swa, fuse_append=True, out_dtype=torch.float32, arrays=False):
     d, t = sc.dims, sc.tables
     h = make_handle(d, out_dtype, sc.cfg.sm_scale)
@@ -461,16 +469,11 @@ def test_prefill_ignores_nonfinite_dead_slots(d, is_swa):
     the cached context, ring slots never written or past the ring's last page, unused pages) hold +inf (K) and NaN
     (V).  Their probabilities are exactly 0, and 0 * NaN must not reach the output through the PV product either
     (Sec. 3.1.3).  Contexts that end inside a 128-key tile, inside a page, and rings that are not full yet."""
-    from helpers import POISON_K, POISON_V
     W, C = d.window, d.ring_slots
     ctx = [0, 1, 5, 63, 64, 65, 100, W - 1, W, W + 1, C - 1, C, C + 7, 1000, 2049]
     q_len = [130, 64, 300, 129, 1, 128, 257, 70, 200, 16, 140, 131, 5, 260, 129]
     sc = build_scenario(d, ctx, q_len, seed=92)
-    pk, pv = wl.bf16_bits_const(POISON_K, (1,))[0], wl.bf16_bits_const(POISON_V, (1,))[0]
-    for pool in (sc.full_pool, sc.swa_pool):
-        assert int((pool[:, 0] == pk).sum()) > 0 and int((pool[:, 1] == pv).sum()) > 0
-        pool[:, 0][pool[:, 0] == pk] = 0x7F80  # +inf
-        pool[:, 1][pool[:, 1] == pv] = 0x7FC0  # NaN
+    poison_dead_slots_nonfinite(sc)
     for fuse_append in (True, False):
         err, lerr = run_prefill(sc, is_swa, fuse_append)
         assert err <= TOL and lerr <= TOL, (fuse_append, err, lerr)
@@ -566,6 +569,49 @@ def test_decode_mtp(d, nq, is_swa):
     assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
     orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
     assert np.array_equal(to_host_bits(pool), ol.pool)
+
+
+@pytest.mark.parametrize("nq", [2, 3, 4])
+def test_decode_mtp_tensor_core_walk(nq):
+    """Full layers at the serving shape (group of 8, head_dim 128, page 64) take the tensor-core multi-token kernel:
+    148 persistent blocks share the flat sequence of 128-key tiles evenly, so a block's slice starts and ends in the
+    middle of (request, KV head) streams and holds several of them.  Contexts from 0 to 40 000 tokens, lengths that
+    end on, just before and just behind tile and page boundaries (the new tokens then straddle two tiles), more
+    requests than one 32-wide scan step, and every dead slot of the pool filled with +inf (K) / NaN (V): outputs
+    and lse against the oracle, pool bytes after the append bit-exact."""
+    d = dims(8, 128, 64, 2)
+    rng = np.random.default_rng(70 + nq)
+    ctx = [40000, 0, 1, 125, 126, 127, 128, 129, 254, 255, 256, 63, 64, 65, 8191, 8192, 8193, 16383, 20000, 3000] + \
+          [int(x) for x in rng.integers(0, 6000, 20)]
+    B = len(ctx)
+    sc = build_scenario(d, ctx, [nq] * B, seed=71 + nq)
+    poison_dead_slots_nonfinite(sc)
+    t = sc.tables
+    h = make_handle(d)
+    pool = to_dev_bf16(sc.full_pool)
+    b = hb.Batch(dev_i32(t.ctx_len), dev_i32(t.block_table), dev_i32(t.ring_table), dev_i32(t.ring_head), None, max_q_len=1,
+                 total_q=B, max_ctx_len=t.max_ctx_len)
+    out = torch.full((B * nq, d.num_q_heads, d.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((B * nq, d.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    need = hb.hswa_decode_workspace_need(h, False, B, t.max_ctx_len, 0, nq)
+    assert 0 < need <= hb.hswa_workspace_bytes(h, B, B * nq, t.max_ctx_len + nq)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    hb.hswa_decode_attn_mtp(h, hb.Layer(pool, False), b, nq, to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new),
+                            out, lse, ws)
+    check_no_async_error(h)
+    ol = sc.layer(False)
+    ref, ref_lse = orc.attention(sc.cfg, ol, sc.batch(), sc.q, sc.k_new, sc.v_new)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.abs(got - ref).max() <= TOL and np.abs(lse.cpu().numpy() - ref_lse).max() <= TOL
+    orc.kv_append(sc.cfg, ol, sc.batch(), sc.k_new, sc.v_new)
+    assert np.array_equal(to_host_bits(pool), ol.pool)
+    # one byte less of workspace than the stated need is refused on the host
+    short = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(hb.HswaError) as e:
+        hb.hswa_decode_attn_mtp(h, hb.Layer(pool, False), b, nq, to_dev_bf16(sc.q), to_dev_bf16(sc.k_new),
+                                to_dev_bf16(sc.v_new), out, lse, short)
+    assert e.value.status == hb.HSWA_ERR_WORKSPACE
 
 
 # ---------------------------------------------------------------------------------------------------------
