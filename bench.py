@@ -175,7 +175,8 @@ class DecodeBench:
         ws_bytes = hb.hswa_workspace_bytes(self.h, B, B * mtp, self.max_ctx)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=device)
         self.full_idx = [i for i, s in enumerate(w.layer_is_swa) if not s]
-        self.launches_per_step = sum(1 if s else (3 if self.shared_prefix else 2) for s in w.layer_is_swa) + 1
+        # kernels per Full layer: decode + combine (+ the shared-prefix stage); with draft tokens: append + decode + combine
+        self.launches_per_step = sum(1 if s else (3 if (self.shared_prefix or mtp > 1) else 2) for s in w.layer_is_swa) + 1
 
     def reset(self):
         self.ctx.copy_(self.ctx0)
@@ -820,8 +821,10 @@ def decode_rooflines(w, bench, m, peaks, steps, warmup, read_gbs, traffic_key=No
     # logical figure (what a sharing-oblivious kernel asks for, partly served by L2) is reported beside it
     ach = ach_u if shared else ach_l
     roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-            "traffic": None, "kernel": "decode_kernel + combine_kernel, one Full layer"
-            + (" (+ prefill_tc_kernel<prefix> with --cascade)" if bench.shared_prefix else ""),
+            "traffic": None,
+            "kernel": ("append_kernel + decode_mtp_tc_kernel + combine_runs_kernel, one Full layer" if bench.mtp > 1 else
+                       "decode_kernel + combine_kernel, one Full layer"
+                       + (" (+ prefill_tc_kernel<prefix> with --cascade)" if bench.shared_prefix else "")),
             "ms_per_launch": ms, "algorithmic_bytes_per_launch": unique if shared else logical,
             "peak_source": peaks["source"] + " (copy: read + write bytes)", "frac_of_nominal_8TBs": ach / 8000.0,
             "frac_of_read_stream": (ach / read_gbs) if read_gbs else None, "read_stream_gbs": read_gbs}
