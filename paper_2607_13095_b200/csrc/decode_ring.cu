@@ -1,13 +1,15 @@
-// SWA-layer decode over the ring of pages, compact-window form (paper Sec. 2.1: an SWA layer attends inside a window
+// SWA-layer decode over the ring of pages, compact-window forms (paper Sec. 2.1: an SWA layer attends inside a window
 // of W keys; Sec. 3.1.1: strictly O(W) KV per request in a ring; Sec. 6.2: a decode step may carry draft tokens).
 //
-// This kernel serves multi-token decode steps on rings longer than the three 64-slot tiles the streaming ring kernel
-// (decode.cu) can keep staged at once; single-token steps and short rings stay on that kernel, which measured faster
-// (12 vs 15 us per layer at batch 64).
+// Two kernels that stage ONLY the 16-slot granules of a ring that meet the window, compactly (72 KB of K and V at
+// W = 128), three blocks per SM; the streaming ring kernel (decode.cu) stages whole 64-slot tiles, two blocks per SM.
+//   decode_ring_window_kernel   single-token steps on batches with more rings than the streaming kernel keeps resident
+//                               (described above the kernel);
+//   decode_ring_compact_kernel  multi-token steps on rings longer than the three tiles the streaming kernel can keep
+//                               staged at once, any window that fits shared memory (described next).
 //
-// Persistent blocks walk (request, KV head) items.  A block stages ONLY the 16-slot granules that meet the window in a
-// compact layout (72 KB of K and V at W = 128), three blocks per SM, and refills the K tiles of its next item as soon as
-// the scores of the current one exist, the V tiles as soon as its output accumulators are complete.
+// decode_ring_compact_kernel: persistent blocks walk (request, KV head) items and refill the K tiles of the next item as
+// soon as the scores of the current one exist, the V tiles as soon as its output accumulators are complete.
 //
 // Work split inside a block (4 warps, no producer / consumer roles):
 //   load      warp 0 works out the circular interval of visible slots [head - min(W - 1, ctx), head + nq - 1] and
@@ -519,6 +521,473 @@ decode_ring_compact_kernel(const __grid_constant__ RingMaps maps, const DecodePa
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Single-token steps, windows up to 128 keys: a loader warp and three compute warps per ring, compact staging.
+//
+// A block owns one (request, KV head) item at a time and stages ONLY the 16-slot granules that meet the window, granule
+// by granule (72 KB of K and V at D = 128), so that three blocks fit an SM; persistent blocks refill their K tiles with
+// the next item's as soon as the scores exist and their V tiles as soon as the output accumulators are complete.
+//   staging  granule-major: a 16-slot granule is [64-column half][16 rows][128 bytes], so that ONE tensor load (5-D
+//            view of the pool, 128-byte swizzle) brings a whole run of granules with both halves of every row.  Issuing
+//            the three or four loads of a K (or V) window costs the issuing warp 1200-1800 cycles, which is why a warp
+//            of its own does nothing else: it waits for "K tiles free" / "V tiles free" and refills them;
+//   scores   split by keys: compute warp c computes S^T[keys x heads] = K Q^T (m16n8k16, the 8 heads of the group are
+//            N) for granules c, c + 3, c + 6 and keeps them in registers; partial maxima meet in shared memory
+//            (named barrier among the compute warps);
+//   softmax  P^T reaches B-fragment order through movmatrix and is left in shared memory, 8 bytes per lane and granule,
+//            for the lane of the same number in every warp; partial row sums beside it (second barrier);
+//   output   split by head dims: a compute warp accumulates O^T[its dims x heads] += V^T P^T over all granules (V^T read
+//            by ldmatrix.trans), so no result has to be merged, and writes its rows from the accumulators (bf16:
+//            transposed once more with movmatrix so that a thread stores two neighbouring dims).
+// One ldmatrix + MMA pair costs a warp about 17 cycles however the code is arranged (the tensor pipe of its scheduler
+// takes one m16n8k16 per 10 cycles); a ring is 144 such pairs.  Fragment loads are issued a granule ahead of the MMAs
+// that use them.
+// Stale rows (slots outside the window, granules not loaded) are masked in the scores and zeroed in the V fragments.
+__device__ __forceinline__ void mma_inorder(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3,
+                                            int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+// Barrier among the three compute warps that also tells every thread whether any of them saw a wait run out, so that
+// all of them leave together (a warp that left alone would leave the others at the next barrier for ever).
+__device__ __forceinline__ bool compute_warps_sync_or(bool failed) {
+  uint32_t any;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q;\n"
+      "setp.ne.u32 q, %1, 0;\n"
+      "bar.red.or.pred p, 1, 96, q;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(any)
+      : "r"((uint32_t)failed)
+      : "memory");
+  return any != 0;
+}
+
+template <int D>
+__global__ void __launch_bounds__(128, 3)
+decode_ring_window_kernel(const __grid_constant__ RingMaps maps, const DecodeParams p, const int n_items) {
+  constexpr int NG = 9;            // granules a window of up to 128 keys can meet: (15 + 127) / 16 + 1
+  constexpr int HALVES = D / 64;
+  constexpr int KS = D / 16;
+  constexpr int NC = 3;                     // compute warps (warps 1 .. 3; warp 0 loads)
+  constexpr int MTOT = D / 16;              // 16-dim output blocks
+  constexpr int MT = (MTOT + NC - 1) / NC;  // per compute warp (the last warp may have fewer)
+  constexpr int KBW = NG / NC;              // granules per compute warp in the score phase
+  constexpr int CHUNKS = D / 8;
+  constexpr int GRAN_BYTES = HALVES * GR * 128;  // one granule of K (or V): [half][16 rows][128 B]
+  constexpr int REGION = NG * GRAN_BYTES;
+  static_assert(2 * CHUNKS <= 32, "one chunk of the new K/V row per lane");
+  static_assert(NG % NC == 0, "granules split evenly over the compute warps");
+  enum { B_KFULL = 0, B_VFULL = 1, B_KFREE = 2, B_VFREE = 3 };
+
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t aK = smem_base, aV = smem_base + REGION;
+  uint8_t* sK = smem;
+  uint8_t* sV = smem + REGION;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * REGION);              // [4]
+  float(*pm)[8] = reinterpret_cast<float(*)[8]>(smem + 2 * REGION + 32);        // [NC] partial row maxima
+  float(*pl)[8] = reinterpret_cast<float(*)[8]>(smem + 2 * REGION + 32 + 128);  // [NC] partial row sums
+  uint2* Pb = reinterpret_cast<uint2*>(smem + 2 * REGION + 32 + 256);           // [NG][32] P^T as B fragments
+  volatile int& s_abort = *reinterpret_cast<volatile int*>(smem + 2 * REGION + 32 + 256 + NG * 256);  // a wait ran out
+
+  const ModelParams& M = p.m;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool fuse = p.k_new != nullptr;
+  const int ring_grans = M.C / GR;
+  const int gpp = M.P / GR;  // granules per page
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars[B_KFULL]), 1);
+    mbar_init(smem_u32(&bars[B_VFULL]), 1);
+    mbar_init(smem_u32(&bars[B_KFREE]), NC);
+    mbar_init(smem_u32(&bars[B_VFREE]), NC);
+    mbar_fence_init();
+    for (int i = 0; i < gpp && i < 4; ++i) tma_prefetch_desc(&maps.m[i]);
+    s_abort = 0;
+  }
+  griddep_launch_dependents();
+  __syncthreads();
+  if (smem_base & 1023u) {  // the swizzled tile addressing assumes a 1 KB-aligned window
+    if (threadIdx.x == 0) record_error(p.err, HSWA_ERR_CUDA, -1, (int)(smem_base & 1023u), 10);
+    return;
+  }
+
+  struct Meta {
+    int ctx, head, my_page;  // lane i keeps page id i of the ring
+  };
+  auto load_meta = [&](int item) {
+    Meta m;
+    const int r = item / M.Hkv;
+    m.ctx = p.b.ctx_len[r];
+    m.head = p.b.ring_head[r];
+    m.my_page = lane < M.R ? p.b.ring_table[(int64_t)r * M.R + lane] : -1;
+    return m;
+  };
+  // A ring head outside [0, C): nothing of such a ring is loaded or written, and the page check records it.  (Applied
+  // where the values are used, so that fetching them ahead does not wait for them.)
+  auto checked = [&](Meta m) {
+    if (m.head < 0 || m.head >= M.C) {
+      m.head = 0;
+      m.my_page = -1;
+    }
+    return m;
+  };
+  // The granules of an item's window: lane i looks after granule i of the visible interval; the first lane of every run
+  // of granules inside one page loads the run (loader warp).  Returns the mask of granules that are (being) loaded,
+  // which every warp works out for itself.
+  auto window_tiles = [&](int item, const Meta& m_raw, int kv, bool issue) -> uint32_t {
+    const Meta m = checked(m_raw);
+    const int r = item / M.Hkv, kh = item % M.Hkv;
+    const int back = min(M.W - 1, max(m.ctx, 0));
+    int start = m.head - back;
+    if (start < 0) start += M.C;
+    const int n_gran = min((start % GR + back) / GR + 1, NG);
+    int gi = start / GR + lane;
+    gi -= gi >= ring_grans ? ring_grans : 0;
+    gi -= gi >= ring_grans ? ring_grans : 0;
+    const int slot_lo = gi * GR;
+    const bool run_start = lane < n_gran && (lane == 0 || gi % gpp == 0);
+    const unsigned starts = __ballot_sync(0xffffffffu, run_start) | (1u << n_gran);
+    const int len = run_start ? __ffs(starts >> (lane + 1)) : 0;
+    const int page = __shfl_sync(0xffffffffu, m.my_page, (slot_lo / M.P) & 31);
+    uint32_t okm = 0;
+    if (run_start) {
+      if (page < 0 || page >= p.num_pages) {
+        if (kv == 0 && issue) record_error(p.err, HSWA_ERR_BOUNDS, r, slot_lo / M.P, page);
+      } else {
+        okm = ((1u << len) - 1u) << lane;
+      }
+    }
+    okm = __reduce_or_sync(0xffffffffu, okm);
+    if (!issue) return okm;
+    const uint32_t full_bar = smem_u32(&bars[kv == 0 ? B_KFULL : B_VFULL]);
+    if (lane == 0) {
+      if (okm == 0)
+        mbar_arrive(full_bar);
+      else
+        mbar_arrive_expect_tx(full_bar, __popc(okm) * GRAN_BYTES);
+    }
+    __syncwarp();
+    if (run_start && ((okm >> lane) & 1u))
+      tma_load_5d((kv == 0 ? aK : aV) + lane * GRAN_BYTES, &maps.m[len - 1], full_bar, 0, 0, 0, (slot_lo % M.P) / GR,
+                  (page * 2 + kv) * M.Hkv + kh);
+    return okm;
+  };
+
+  const int stride = gridDim.x;
+  if (blockIdx.x >= n_items) return;
+  if (warp == 0) {
+    // ---------------- loader warp ----------------
+    int it = blockIdx.x;
+    Meta m_cur = load_meta(it);
+    Meta m_nxt = m_cur;
+    if (it + stride < n_items) m_nxt = load_meta(it + stride);
+    window_tiles(it, m_cur, 0, true);
+    window_tiles(it, m_cur, 1, true);
+    for (int k = 0; it + stride < n_items; ++k, it += stride) {
+      const int par = k & 1;
+      const int nxt = it + stride;
+      m_cur = m_nxt;
+      if (nxt + stride < n_items) m_nxt = load_meta(nxt + stride);
+      // K tiles of item k are dead once every compute warp has its scores, the V tiles once it has its accumulators
+      bool ok = mbar_wait(smem_u32(&bars[B_KFREE]), par);
+      bool k_issued = false;
+      if (ok && !s_abort) {
+        window_tiles(nxt, m_cur, 0, true);
+        k_issued = true;
+        ok = mbar_wait(smem_u32(&bars[B_VFREE]), par);
+        if (ok && !s_abort) window_tiles(nxt, m_cur, 1, true);
+      }
+      if (!ok || s_abort) {
+        // the compute warps gave up, or a wait of this warp ran out: leave once no load of this block is in flight
+        if (!ok && lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, it / M.Hkv, it % M.Hkv, 12);
+        s_abort = 1;
+        mbar_wait(smem_u32(&bars[B_KFULL]), par, 2000000);
+        mbar_wait(smem_u32(&bars[B_VFULL]), par, 2000000);
+        if (k_issued) mbar_wait(smem_u32(&bars[B_KFULL]), par ^ 1, 2000000);
+        return;
+      }
+    }
+    return;
+  }
+
+  // ---------------- compute warps ----------------
+  const int cw = warp - 1;
+  const int g_row = lane >> 2;
+  const int qd = (lane & 3) * 2;
+  const int mi = lane >> 3, mr = lane & 7;
+  uint32_t qf[KS][2];
+  uint4 newrow = make_uint4(0, 0, 0, 0);
+  auto load_q = [&](int item) {
+    const int r = item / M.Hkv, kh = item % M.Hkv;
+    const bool live = g_row < M.G;
+    const __nv_bfloat16* qrow = p.q + ((int64_t)r * M.Hq + kh * M.G + (live ? g_row : 0)) * D;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      qf[ks][0] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd) : 0u;
+      qf[ks][1] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + qd + 8) : 0u;
+    }
+    if (fuse && lane < 2 * CHUNKS)
+      newrow = *reinterpret_cast<const uint4*>((lane < CHUNKS ? p.k_new : p.v_new) + ((int64_t)r * M.Hkv + kh) * D +
+                                               (lane % CHUNKS) * 8);
+  };
+  // Byte offset of 16-byte chunk c (0 .. CHUNKS - 1) of row jr (0 .. 15) inside a granule
+  auto gran_off = [](int jr, int c) { return (uint32_t)((c >> 3) * (GR * 128)) + swz128(jr, c & 7); };
+  // This thread's ldmatrix row addresses inside a granule: K fragments of k-step ks, V^T fragments of this warp's dim
+  // blocks cw * MT + mt
+  uint32_t k_off[KS], v_off[MT];
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) k_off[ks] = gran_off((mi & 1) * 8 + mr, 2 * ks + (mi >> 1));
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) v_off[mt] = gran_off((mi >> 1) * 8 + mr, (2 * (cw * MT + mt) + (mi & 1)) % CHUNKS);
+  const int n_mt = min(MT, MTOT - cw * MT);  // dim blocks of this warp (warp-uniform)
+
+  int it = blockIdx.x;
+  // lengths, ring heads and ring tables are fetched two items ahead: right behind the dependency wait such a fetch
+  // takes a few thousand cycles, more than the first item's scores
+  Meta mt_next = load_meta(it);
+  Meta mt_next2 = mt_next;
+  if (it + stride < n_items) mt_next2 = load_meta(it + stride);
+  uint32_t okm_next = window_tiles(it, mt_next, 0, false);
+  griddep_wait();  // q, k_new, v_new and the outputs may belong to the previous kernel until here
+  load_q(it);
+
+  for (int k = 0; it < n_items; ++k, it += stride) {
+    const int par = k & 1;
+    const int r = it / M.Hkv, kh = it % M.Hkv;
+    const Meta m = checked(mt_next);
+    const uint32_t okm = okm_next;
+    const int nxt = it + stride;
+    const bool has_next = nxt < n_items;
+    mt_next = mt_next2;
+    if (nxt + stride < n_items) mt_next2 = load_meta(nxt + stride);
+    const int back = min(M.W - 1, max(m.ctx, 0));  // cached positions the new token can see
+    int start = m.head - back;                      // ring slot of the oldest visible position
+    if (start < 0) start += M.C;
+    const int sr = start % GR;
+    const int hi_row = sr + back;                   // compact row of the new token; visible rows are [sr, hi_row]
+    const int n_gran = min(hi_row / GR + 1, NG);
+    auto visible = [&](int j) { return ((okm >> (j / GR)) & 1u) && j >= sr && j <= hi_row; };
+    auto interior = [&](int kb) { return ((okm >> kb) & 1u) && kb * 16 >= sr && kb * 16 + 15 <= hi_row; };
+
+    // A wait that ran out: the warp still reaches the next barrier among the compute warps, where all of them learn
+    // of it and leave (the flag tells the loader warp, which outwaits the loads the block still has in flight).
+    bool failed = false;
+    if (!mbar_wait(smem_u32(&bars[B_KFULL]), par)) {
+      failed = true;
+      s_abort = 1;
+      if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, kh, 10);
+    }
+    // every warp patches the new K row itself (same bytes), so that it needs no barrier before reading it
+    if (fuse && lane < CHUNKS) {
+      *reinterpret_cast<uint4*>(sK + (hi_row >> 4) * GRAN_BYTES + gran_off(hi_row & 15, lane)) = newrow;
+      fence_proxy_async_smem();  // a later TMA load overwrites this row
+    }
+    __syncwarp();
+
+    // ---------------- scores of granules cw, cw + NC, ... ----------------
+    float s[KBW][4];
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+    {
+      uint32_t ka[2][KS][4];
+      if (cw < n_gran) {
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+          ldmatrix_x4(aK + cw * GRAN_BYTES + k_off[ks], ka[0][ks][0], ka[0][ks][1], ka[0][ks][2], ka[0][ks][3]);
+      }
+#pragma unroll
+      for (int i = 0; i < KBW; ++i) {
+        const int kb = cw + NC * i;
+        if (kb < n_gran) {
+          if (i + 1 < KBW && kb + NC < n_gran) {
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks)
+              ldmatrix_x4(aK + (kb + NC) * GRAN_BYTES + k_off[ks], ka[(i + 1) & 1][ks][0], ka[(i + 1) & 1][ks][1],
+                          ka[(i + 1) & 1][ks][2], ka[(i + 1) & 1][ks][3]);
+          }
+          float e[4] = {0.f, 0.f, 0.f, 0.f}, f[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int ks = 0; ks < KS; ++ks) mma_inorder((ks & 1) ? f : e, ka[i & 1][ks], qf[ks][0], qf[ks][1]);
+          const int keyA = kb * 16 + g_row, keyB = keyA + 8;
+          const bool inner = interior(kb);
+          const bool vA = inner || visible(keyA), vB = inner || visible(keyB);
+          s[i][0] = vA ? (e[0] + f[0]) * M.scale_log2 : -INFINITY;
+          s[i][1] = vA ? (e[1] + f[1]) * M.scale_log2 : -INFINITY;
+          s[i][2] = vB ? (e[2] + f[2]) * M.scale_log2 : -INFINITY;
+          s[i][3] = vB ? (e[3] + f[3]) * M.scale_log2 : -INFINITY;
+        } else {
+          s[i][0] = s[i][1] = s[i][2] = s[i][3] = -INFINITY;
+        }
+        mx0 = fmaxf(mx0, fmaxf(s[i][0], s[i][2]));
+        mx1 = fmaxf(mx1, fmaxf(s[i][1], s[i][3]));
+      }
+    }
+    __syncwarp();  // every lane's K fragments are in registers
+    if (lane == 0) mbar_arrive(smem_u32(&bars[B_KFREE]));
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+    }
+    if (lane < 4) {
+      pm[cw][qd] = mx0;
+      pm[cw][qd + 1] = mx1;
+    }
+    // the cache copy of the new row (last compute warp: K from lanes [0, CHUNKS), V from lanes [CHUNKS, 2 CHUNKS))
+    const uint4 vrow = newrow;
+    const int new_page = __shfl_sync(0xffffffffu, m.my_page, (m.head / M.P) & 31);
+    if (fuse && cw == NC - 1 && lane < 2 * CHUNKS && !failed) {
+      const int kv = lane / CHUNKS, ch = lane % CHUNKS;
+      if (new_page < 0 || new_page >= p.num_pages) {
+        if (lane == 0) record_error(p.err, HSWA_ERR_BOUNDS, r, -1, new_page);
+      } else {
+        *reinterpret_cast<uint4*>(p.pool + ((((int64_t)new_page * 2 + kv) * M.Hkv + kh) * M.P + m.head % M.P) * D + ch * 8) =
+            newrow;
+      }
+    }
+    if (has_next) {
+      load_q(nxt);  // consumed an iteration from now
+      okm_next = window_tiles(nxt, mt_next, 0, false);
+    }
+    if (compute_warps_sync_or(failed)) return;  // barrier 1: every partial maximum is published
+
+    // ---------------- softmax of this warp's granules: P^T as B fragments, partial row sums ----------------
+    mx0 = fmaxf(fmaxf(pm[0][qd], pm[1][qd]), pm[2][qd]);
+    mx1 = fmaxf(fmaxf(pm[0][qd + 1], pm[1][qd + 1]), pm[2][qd + 1]);
+    const float m0 = mx0 == -INFINITY ? 0.f : mx0, m1 = mx1 == -INFINITY ? 0.f : mx1;
+    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < KBW; ++i) {
+      const int kb = cw + NC * i;
+      // bf16 values the tensor core will multiply; the row sums add exactly those
+      const uint32_t lo = pack_bf16x2(fast_exp2(s[i][0] - m0), fast_exp2(s[i][1] - m1));  // key g_row: heads qd, qd + 1
+      const uint32_t hi = pack_bf16x2(fast_exp2(s[i][2] - m0), fast_exp2(s[i][3] - m1));  // key g_row + 8
+      const float2 flo = unpack_bf16x2(lo), fhi = unpack_bf16x2(hi);
+      l0 += flo.x + fhi.x;
+      l1 += flo.y + fhi.y;
+      const uint32_t b0 = movmatrix_trans(lo);  // keys 2t, 2t + 1 of head g_row
+      const uint32_t b1 = movmatrix_trans(hi);  // keys 2t + 8, 2t + 9
+      Pb[kb * 32 + lane] = make_uint2(b0, b1);
+    }
+#pragma unroll
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+    }
+    if (lane < 4) {
+      pl[cw][qd] = l0;
+      pl[cw][qd + 1] = l1;
+    }
+
+    // ---------------- output: this warp's head dims over all granules ----------------
+    if (!mbar_wait(smem_u32(&bars[B_VFULL]), par)) {
+      failed = true;
+      s_abort = 1;
+      if (lane == 0) record_error(p.err, HSWA_ERR_TIMEOUT, r, kh, 11);
+    }
+    if (fuse && lane >= CHUNKS && lane < 2 * CHUNKS) {
+      *reinterpret_cast<uint4*>(sV + (hi_row >> 4) * GRAN_BYTES + gran_off(hi_row & 15, lane - CHUNKS)) = vrow;
+      fence_proxy_async_smem();
+    }
+    if (compute_warps_sync_or(failed)) return;  // barrier 2: P and the partial sums are complete
+    float o[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    {
+      uint32_t va[2][MT][4];
+      uint2 pbv[2];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+        if (mt < n_mt) ldmatrix_x4_trans(aV + v_off[mt], va[0][mt][0], va[0][mt][1], va[0][mt][2], va[0][mt][3]);
+      pbv[0] = Pb[lane];
+#pragma unroll
+      for (int kb = 0; kb < NG; ++kb) {
+        if (kb < n_gran) {
+          if (kb + 1 < NG && kb + 1 < n_gran) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+              if (mt < n_mt)
+                ldmatrix_x4_trans(aV + (kb + 1) * GRAN_BYTES + v_off[mt], va[(kb + 1) & 1][mt][0], va[(kb + 1) & 1][mt][1],
+                                  va[(kb + 1) & 1][mt][2], va[(kb + 1) & 1][mt][3]);
+            pbv[(kb + 1) & 1] = Pb[(kb + 1) * 32 + lane];
+          }
+          // V^T fragments: a0 / a1 hold keys 16 kb + qd, qd + 1 in their halves, a2 / a3 keys 16 kb + 8 + qd, qd + 9.
+          // Rows outside the window may hold anything: zero them (0 x NaN would poison the sum).
+          if (!interior(kb)) {
+            const int k0 = kb * 16 + qd;
+            const uint32_t keep_lo = (visible(k0) ? 0x0000ffffu : 0u) | (visible(k0 + 1) ? 0xffff0000u : 0u);
+            const uint32_t keep_hi = (visible(k0 + 8) ? 0x0000ffffu : 0u) | (visible(k0 + 9) ? 0xffff0000u : 0u);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+              va[kb & 1][mt][0] &= keep_lo;
+              va[kb & 1][mt][1] &= keep_lo;
+              va[kb & 1][mt][2] &= keep_hi;
+              va[kb & 1][mt][3] &= keep_hi;
+            }
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            if (mt < n_mt) mma_inorder(o[mt], va[kb & 1][mt], pbv[kb & 1].x, pbv[kb & 1].y);
+        }
+      }
+    }
+    // row sums of this thread's accumulator columns (heads qd, qd + 1), read before the next item may overwrite them
+    l0 = pl[0][qd] + pl[1][qd] + pl[2][qd];
+    l1 = pl[0][qd + 1] + pl[1][qd + 1] + pl[2][qd + 1];
+    __syncwarp();  // this warp is done with the V tiles
+    if (lane == 0) mbar_arrive(smem_u32(&bars[B_VFREE]));
+
+    const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
+    if (M.out_fp32) {
+      // thread: heads qd, qd + 1; head dims 16 (cw MT + mt) + g_row and + 8 (eight lanes fill a 32-byte sector)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        if (qd + j >= M.G) continue;
+        const float inv = j ? inv1 : inv0;
+        float* orow = reinterpret_cast<float*>(p.out) + ((int64_t)r * M.Hq + kh * M.G + qd + j) * D + cw * MT * 16 + g_row;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          if (mt < n_mt) {
+            orow[mt * 16] = o[mt][j] * inv;
+            orow[mt * 16 + 8] = o[mt][2 + j] * inv;
+          }
+        }
+      }
+    } else {
+      // transposed once more: the thread then holds head g_row, dims 16 (cw MT + mt) + qd, qd + 1 (and + 8) as bf16 pairs
+      __nv_bfloat16* orow =
+          reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)r * M.Hq + kh * M.G + g_row) * D + cw * MT * 16 + qd;
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const uint32_t w0 = movmatrix_trans(pack_bf16x2(o[mt][0] * inv0, o[mt][1] * inv1));
+        const uint32_t w1 = movmatrix_trans(pack_bf16x2(o[mt][2] * inv0, o[mt][3] * inv1));
+        if (g_row < M.G && mt < n_mt) {
+          *reinterpret_cast<uint32_t*>(orow + mt * 16) = w0;
+          *reinterpret_cast<uint32_t*>(orow + mt * 16 + 8) = w1;
+        }
+      }
+    }
+    if (p.lse && cw == 0 && g_row == 0) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        if (qd + j >= M.G) continue;
+        const float l = j ? l1 : l0, mm = j ? mx1 : mx0;
+        p.lse[(int64_t)r * M.Hq + kh * M.G + qd + j] = l > 0.f ? (mm + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      }
+    }
+  }
+}
+
 struct CompactPlan {
   int ng_max, k_region, smem;
 };
@@ -583,6 +1052,60 @@ bool hswa_ring_compact_supported(const ModelParams& m, int nq) {
   return c.ng_max <= 31 && c.smem <= 200 * 1024;
 }
 
+// 5-D views of the pool {64, 16, D / 64, P / 16, num_pages * 2 * Hkv}: a box {64, 16, D / 64, k, 1} is a run of k granules
+// of one (page, K|V, head) slab, landing granule by granule with the two 64-column halves of a granule behind each other.
+cudaError_t make_ring_maps5(const hswa_handle* h, const DecodeParams& p, RingMaps* out) {
+  const ModelParams& m = p.m;
+  const int halves = m.D / 64, gpp = m.P / GR;
+  cuuint64_t dims[5] = {64, (cuuint64_t)GR, (cuuint64_t)halves, (cuuint64_t)gpp, (cuuint64_t)p.num_pages * 2 * m.Hkv};
+  cuuint64_t strides[4] = {(cuuint64_t)m.D * 2, 128, (cuuint64_t)GR * m.D * 2, (cuuint64_t)m.P * m.D * 2};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < 4; ++i) {
+    const int k = i + 1 <= gpp ? i + 1 : 1;  // runs longer than a page do not exist
+    cuuint32_t box[5] = {64, (cuuint32_t)GR, (cuuint32_t)halves, (cuuint32_t)k, 1};
+    if (h->encode_tiled(&out->m[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, p.pool, dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  return cudaSuccess;
+}
+
+// Can the compact single-token kernel serve this shape?  (The window's granules, at most nine, stay in registers as scores.)
+bool hswa_ring_window_supported(const ModelParams& m, int nq) {
+  return nq == 1 && m.W <= 128 && m.P % GR == 0 && (m.D == 64 || m.D == 128) && m.G <= 8 && m.R <= 32;
+}
+
+cudaError_t hswa_launch_decode_ring_window(const hswa_handle* h, const DecodeParams& p, bool early_start, cudaStream_t s) {
+  if (p.b.B == 0) return cudaSuccess;
+  RingMaps maps;
+  cudaError_t e = make_ring_maps5(h, p, &maps);
+  if (e != cudaSuccess) return e;
+  const int D = p.m.D;
+  const int smem = 2 * (D / 64) * 9 * GR * 128 + 32 + 256 + 9 * 256 + 16;  // K and V granules, barriers, maxima / sums, P, flag
+  auto kern = D == 128 ? decode_ring_window_kernel<128> : decode_ring_window_kernel<64>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  // three blocks fit an SM only with the whole unified cache configured as shared memory
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  const int n_items = p.b.B * p.m.Hkv;
+  int per_sm = (228 * 1024) / (smem + 1024);
+  if (per_sm > 4) per_sm = 4;
+  const int resident = h->num_sms * per_sm;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_items < resident ? n_items : resident, 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, maps, p, n_items);
+}
+
 cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
                                             bool early_start, cudaStream_t s) {
   if (p.b.B == 0) return cudaSuccess;
@@ -601,3 +1124,4 @@ cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensor
   if (D == 64 && NT == 4) return launch_compact_t<64, 4>(maps, p, c, h->num_sms, early_start, s);
   return cudaErrorInvalidValue;
 }
+

@@ -126,6 +126,9 @@ cudaError_t hswa_launch_combine(const DecodeParams& p, cudaStream_t s);
 bool hswa_ring_compact_supported(const ModelParams& m, int nq);
 cudaError_t hswa_launch_decode_ring_compact(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
                                             bool early_start, cudaStream_t s);
+// SWA layers, one new token, windows up to 128 keys: one autonomous warp per (request, KV head)
+bool hswa_ring_window_supported(const ModelParams& m, int nq);
+cudaError_t hswa_launch_decode_ring_window(const hswa_handle* h, const DecodeParams& p, bool early_start, cudaStream_t s);
 cudaError_t hswa_launch_decode_mtp(const hswa_handle* h, const CUtensorMap& tm_pool, const DecodeParams& p,
                                    bool early_start, cudaStream_t s);
 // Multi-token decode on Full layers on the tensor cores (group of 8, head_dim 128, page 64, 2-4 tokens per request)

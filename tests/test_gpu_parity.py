@@ -124,6 +124,27 @@ def test_decode_sweep(d, is_swa):
         assert err <= TOL and lerr <= TOL, (fused, err, lerr)
 
 
+@pytest.mark.parametrize("d", [dims(8, 128, 64), dims(4, 64, 16, 1), dims(3, 64, 32, 2, W=33), dims(5, 128, 32, 3, W=100),
+                               dims(8, 128, 16, 2, W=128)], ids=str)
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_decode_swa_many_rings(d, out_dtype):
+    """SWA decode on batches with more rings than three per SM: the compact single-token kernel serves them, and some
+    of its blocks walk a second ring.  Contexts cross every window / page / ring boundary, ring heads are random,
+    every dead slot holds +inf / NaN; with and without the fused append; fp32 and bf16 output (the bf16 result is the
+    fp32 one rounded once: half a bf16 ulp on top of the bar)."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    B = (3 * sms + 40 + d.num_kv_heads - 1) // d.num_kv_heads
+    W, P, C = d.window, d.page_size, d.ring_slots
+    base = [0, 1, 2, 15, 16, 17, W - 2, W - 1, W, W + 1, P - 1, P, P + 1, C - 1, C, C + 1, 2 * C + 5, 300, 517]
+    ctx = [base[i % len(base)] + (i // len(base)) % 3 for i in range(B)]
+    sc = build_scenario(d, ctx, [1] * B, seed=23)
+    poison_dead_slots_nonfinite(sc)
+    tol = TOL if out_dtype == torch.float32 else 2 * TOL
+    for fused in (True, False):
+        err, lerr = run_decode(sc, True, fused, out_dtype=out_dtype)
+        assert err <= tol and lerr <= TOL, (fused, err, lerr)
+
+
 def test_decode_long_split_and_bf16_out():
     d = dims(8, 128, 64, 2)
     sc = build_scenario(d, [40000, 9000, 33, 20481], [1, 1, 1, 1], seed=9)
