@@ -1177,8 +1177,8 @@ cudaError_t hswa_launch_decode(const hswa_handle* h, const CUtensorMap& tm_pool,
     // stage buffers at once, so longer rings take the compact-window kernel
     if (p.nq > 1 && (p.m.C + TK - 1) / TK > 3) return hswa_launch_decode_ring_compact(h, tm_pool, p, early_start, s);
     // single-token steps with more rings than the streaming kernel keeps resident (two blocks per SM): the compact
-    // kernel holds three rings per SM and loses one round of the walk (17 vs 21 us per layer at batch 128, 12.1 vs 12.5
-    // at batch 64; on fewer rings the streaming kernel's shorter path per ring wins, 5.3 vs 5.6 us at batch 16)
+    // kernel holds three or four rings per SM and loses a round of the walk (17 vs 21 us per layer at batch 128, 10.9 vs
+    // 12.5 at batch 64; on fewer rings the streaming kernel's shorter path per ring wins, 5.3 vs 5.6 us at batch 16)
     if (p.b.B * p.m.Hkv > 2 * h->num_sms && hswa_ring_window_supported(p.m, p.nq))
       return hswa_launch_decode_ring_window(h, p, early_start, s);
     if (D == 128 && P == 64) return launch_ring_t<128, 64>(h, tm_pool, p, early_start, s);

@@ -127,13 +127,15 @@ def test_decode_sweep(d, is_swa):
 @pytest.mark.parametrize("d", [dims(8, 128, 64), dims(4, 64, 16, 1), dims(3, 64, 32, 2, W=33), dims(5, 128, 32, 3, W=100),
                                dims(8, 128, 16, 2, W=128)], ids=str)
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-def test_decode_swa_many_rings(d, out_dtype):
-    """SWA decode on batches with more rings than three per SM: the compact single-token kernel serves them, and some
-    of its blocks walk a second ring.  Contexts cross every window / page / ring boundary, ring heads are random,
-    every dead slot holds +inf / NaN; with and without the fused append; fp32 and bf16 output (the bf16 result is the
-    fp32 one rounded once: half a bf16 ulp on top of the bar)."""
+@pytest.mark.parametrize("n_per_sm", [3, 4], ids=["over3", "over4"])
+def test_decode_swa_many_rings(d, out_dtype, n_per_sm):
+    """SWA decode on batches with more rings than three (four) per SM: the compact single-token kernel serves them --
+    between three and four per SM at head_dim 128 in its form with four blocks per SM, whose late V granules take the K
+    area -- and some of its blocks walk a second ring.  Contexts cross every window / page / ring boundary, ring heads
+    are random, every dead slot holds +inf / NaN; with and without the fused append; fp32 and bf16 output (the bf16
+    result is the fp32 one rounded once: half a bf16 ulp on top of the bar)."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    B = (3 * sms + 40 + d.num_kv_heads - 1) // d.num_kv_heads
+    B = (n_per_sm * sms + 40 + d.num_kv_heads - 1) // d.num_kv_heads
     W, P, C = d.window, d.page_size, d.ring_slots
     base = [0, 1, 2, 15, 16, 17, W - 2, W - 1, W, W + 1, P - 1, P, P + 1, C - 1, C, C + 1, 2 * C + 5, 300, 517]
     ctx = [base[i % len(base)] + (i // len(base)) % 3 for i in range(B)]
