@@ -181,9 +181,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
   // its neighbours: a warp that skipped phases could pass a barrier that is still one fill behind.
   static_assert(NS % NW == 0, "a stage must always be consumed by the same warp");
 
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * NS];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // All shared memory is one dynamic window (no static part, so that it starts on the 1 KB boundary the swizzled tiles
+  // need without slack): the stage buffers, then the barriers.
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NS * STAGE_BYTES);  // [2 * NS]
   const uint32_t smem_base = smem_u32(smem);
 
   const int r = blockIdx.x, split = blockIdx.y, kh = blockIdx.z;
@@ -221,6 +222,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_pool, const DecodeParams p)
     }
     mbar_fence_init();
     tma_prefetch_desc(&tm_pool);
+    if (smem_base & 1023u) record_error(p.err, HSWA_ERR_CUDA, -1, (int)(smem_base & 1023u), 15);  // tiles would be misread
   }
   __syncthreads();
 
@@ -1148,7 +1150,7 @@ cudaError_t launch_mtp_t(const CUtensorMap& tm, const DecodeParams& p, cudaStrea
 template <int D, int P, int NS, int NW>
 cudaError_t launch_decode_t(const CUtensorMap& tm, const DecodeParams& p, bool early_start, cudaStream_t s) {
   constexpr int STAGE_BYTES = 2 * (D / 64) * TK * 128;
-  constexpr int SMEM = NS * STAGE_BYTES + 1024;
+  constexpr int SMEM = NS * STAGE_BYTES + 2 * NS * 8 + 16;  // stage buffers, barriers
   static_assert(NW * 8 * D * 4 + NW * 64 <= NS * STAGE_BYTES, "merge scratch must fit the stage buffers");
   auto kern = decode_kernel<D, P, NS, NW>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);

@@ -42,10 +42,8 @@ constexpr int REGS_SERVICE = 56, REGS_SOFTMAX = 224;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                  // 2 Q tiles
-constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;             // KV_STAGES K tiles
-constexpr int OFF_V = OFF_K + KV_STAGES * TILE_BYTES;     // KV_STAGES V tiles
-constexpr int SMEM_TILES = OFF_V + KV_STAGES * TILE_BYTES;  // 196608
-constexpr int SMEM_BYTES = SMEM_TILES + 1024;
+constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;             // the K ring, then the V ring (both `stages` tiles deep)
+constexpr int tile_kernel_smem(int stages) { return OFF_K + 2 * stages * TILE_BYTES + 256; }  // + barriers and flags
 
 constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_PV = IDESC_S | (1u << 16);  // B (= V) is MN-major: [key][d] with d contiguous
@@ -229,17 +227,23 @@ __device__ __forceinline__ void linger_after_error(const int32_t* err) {
 // never written, or past the ring's last page).
 __device__ __forceinline__ bool v_tile_needs_patch(int is_swa, int ctx, int j) { return is_swa || ctx - j * BN < BN; }
 
-template <bool PREFIX>
+// STAGES = depth of the K and of the V tile ring: 2 for prefill; 1 for the shared-prefix stage, whose block then leaves
+// room on its SM for a block of the suffix decode kernel that streams beside it.
+template <bool PREFIX, int STAGES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_constant__ CUtensorMap tm_q,
                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                   const PrefillParams p, const int max_tiles) {  // tiles b < max_tiles only
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[NUM_BARS];
-  __shared__ uint32_t tmem_base_slot;
-  __shared__ int mma_abort;  // set by an MMA issuer that gave up, read by the other one
-  __shared__ int picked[2];  // (request, tile) of this block under the longest-first order; request -1: none
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // All shared memory is one dynamic window (no static part, so that it starts on the 1 KB boundary the swizzled tiles
+  // need without slack): Q tiles | K ring | V ring | barriers and flags.
+  extern __shared__ __align__(1024) uint8_t smem[];
+  constexpr int OFF_V = OFF_K + STAGES * TILE_BYTES;
+  constexpr int OFF_STATE = OFF_V + STAGES * TILE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_STATE);                     // [NUM_BARS]
+  uint32_t& tmem_base_slot = *reinterpret_cast<uint32_t*>(smem + OFF_STATE + 160);
+  int& mma_abort = *reinterpret_cast<int*>(smem + OFF_STATE + 164);  // set by an MMA issuer that gave up, read by the other
+  int* picked = reinterpret_cast<int*>(smem + OFF_STATE + 168);      // [2] (request, tile) under the longest-first order
+  static_assert(NUM_BARS * 8 <= 160, "barriers fit their slot");
   const uint32_t sbase = smem_u32(smem);
   const ModelParams& M = p.m;
 
@@ -302,7 +306,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
   }
   // An earlier block gave up: do not queue behind it.  One thread reads the error word so that the whole block
   // takes the same decision (the MMA issuers below wait for each other on counted barriers).
-  if (threadIdx.x == 0) mma_abort = *reinterpret_cast<volatile int32_t*>(p.err) != 0;
+  if (threadIdx.x == 0) {
+    mma_abort = *reinterpret_cast<volatile int32_t*>(p.err) != 0;
+    if (sbase & 1023u) {  // the swizzled tile addressing assumes a 1 KB-aligned window
+      record_error(p.err, HSWA_ERR_CUDA, -1, (int)(sbase & 1023u), 14);
+      mma_abort = 1;
+    }
+  }
   __syncthreads();
   if (mma_abort) return;
   const int n_tiles = seq.total();
@@ -314,7 +324,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
 
   if (threadIdx.x == 0) {
     mbar_init(bar(BAR_Q), 1);
-    for (int s = 0; s < KV_STAGES; ++s) {
+    for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar(BAR_KFULL + s), 1);
       mbar_init(bar(BAR_KEMPTY + s), 2);  // one commit per MMA issuer
       mbar_init(bar(BAR_VFULL + s), 1);
@@ -326,7 +336,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     }
     mbar_init(bar(BAR_OFINAL), 1);
     mbar_init(bar(BAR_OFINAL + 1), 1);
-    static_assert(KV_STAGES == 2, "one patch barrier per V stage");
+    static_assert(STAGES <= 2, "one patch barrier per V stage");
     mbar_init(bar(BAR_VPATCH), 1);
     mbar_init(bar(BAR_VPATCH + 1), 1);
     mbar_fence_init();
@@ -368,7 +378,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
     int pid_cur = 0;
     bool ok = true;
     for (int j = 0; j < n_tiles && ok; ++j) {
-      const int stage = j % KV_STAGES;
+      const int stage = j % STAGES;
       int pg[2] = {0, 0};
       // Rows of a cached tile that no row of this block can see (the tail of the last page of a Full layer; ring
       // slots never written, past the ring's last page, or older than the first row's window, which a ring seeded
@@ -390,11 +400,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       if (lane == 0) {
         // K and V slots are released separately (K right after the S MMAs that read it, V only after both tiles'
         // PV MMAs), so each load waits for its own slot: the K tile is on its way a whole step earlier.
-        const uint32_t par = ((j / KV_STAGES) - 1) & 1;
+        const uint32_t par = ((j / STAGES) - 1) & 1;
         const uint32_t dK = sbase + OFF_K + stage * TILE_BYTES, dV = sbase + OFF_V + stage * TILE_BYTES;
         for (int kv = 0; kv < 2 && ok; ++kv) {
           const uint32_t full_mma = bar((kv ? BAR_VFULL : BAR_KFULL) + stage);
-          if (j >= KV_STAGES && !mbar_wait(bar((kv ? BAR_VEMPTY : BAR_KEMPTY) + stage), par)) {
+          if (j >= STAGES && !mbar_wait(bar((kv ? BAR_VEMPTY : BAR_KEMPTY) + stage), par)) {
             record_error(p.err, HSWA_ERR_TIMEOUT, r, j, 10 + kv);
             ok = false;
             break;
@@ -478,11 +488,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       token_pass();
       bool done = !ok || *abort_flag != 0;
       for (int j = 0; j < n_tiles && !done; ++j) {
-        const int stage = j % KV_STAGES, nstage = (j + 1) % KV_STAGES;
+        const int stage = j % STAGES, nstage = (j + 1) % STAGES;
         const bool more = j + 1 < n_tiles;
         // polled during the other issuer's turn
-        ok = mbar_wait(bar(BAR_VFULL + stage), (j / KV_STAGES) & 1) && mbar_wait(bar(BAR_PFULL + P_PARTS * i), j & 1);
-        if (ok && more) ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / KV_STAGES) & 1);
+        ok = mbar_wait(bar(BAR_VFULL + stage), (j / STAGES) & 1) && mbar_wait(bar(BAR_PFULL + P_PARTS * i), j & 1);
+        if (ok && more) ok = mbar_wait(bar(BAR_KFULL + nstage), ((j + 1) / STAGES) & 1);
         token_wait();
         if (!ok) *abort_flag = 1;
         if (*abort_flag != 0) {
@@ -520,7 +530,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_pool, const __grid_cons
       uint32_t n_patched = 0;  // bit s: parity of the next patch of stage s
       for (int j = 0; j < seq.nA; ++j) {
         if (!v_tile_needs_patch(p.is_swa, ctx, j)) continue;
-        const int stage = j % KV_STAGES;
+        const int stage = j % STAGES;
         // the producer arms this barrier once per patched tile of the stage, after the stage's previous tile has been
         // consumed: this warp sees each of its phases in turn
         if (!mbar_wait(bar(BAR_VPATCH + stage), (n_patched >> stage) & 1u)) {
@@ -1523,14 +1533,16 @@ cudaError_t hswa_launch_prefill_swa_packed(const CUtensorMap& tm_q, const CUtens
 cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                    const CUtensorMap& tm_v, const PrefillParams& p, int tile_limit, cudaStream_t s) {
   if (p.b.B == 0 || p.total_q == 0 || p.max_q_len == 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  constexpr int SMEM_BYTES = tile_kernel_smem(KV_STAGES);
+  auto kern = prefill_tc_kernel<false, KV_STAGES>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  static const cudaError_t budget = check_register_budget(prefill_tc_kernel<false>, NUM_THREADS);
+  static const cudaError_t budget = check_register_budget(kern, NUM_THREADS);
   if (budget != cudaSuccess) return budget;
   int max_tiles = (p.max_q_len + BM - 1) / BM;
   if (tile_limit > 0 && tile_limit < max_tiles) max_tiles = tile_limit;
   dim3 grid(p.m.G / 2, p.m.Hkv, (unsigned)(p.b.B * max_tiles));
-  prefill_tc_kernel<false><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
+  kern<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_k, tm_v, p, max_tiles);
   return cudaGetLastError();
 }
 
@@ -1540,12 +1552,17 @@ cudaError_t hswa_launch_prefill_tc(const CUtensorMap& tm_pool, const CUtensorMap
 cudaError_t hswa_launch_decode_prefix(const CUtensorMap& tm_pool, const CUtensorMap& tm_q, const PrefillParams& p,
                                       int n_slices, cudaStream_t s) {
   if (p.b.B == 0 || n_slices <= 0) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  constexpr int PREFIX_STAGES = KV_STAGES;
+  constexpr int SMEM_BYTES = tile_kernel_smem(PREFIX_STAGES);
+  auto kern = prefill_tc_kernel<true, PREFIX_STAGES>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  static const cudaError_t budget = check_register_budget(prefill_tc_kernel<true>, NUM_THREADS);
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  static const cudaError_t budget = check_register_budget(kern, NUM_THREADS);
   if (budget != cudaSuccess) return budget;
   dim3 grid(n_slices, p.m.Hkv, (p.b.B + 31) / 32);
-  prefill_tc_kernel<true><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_pool, tm_pool, p, 1);
+  kern<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tm_pool, tm_q, tm_pool, tm_pool, p, 1);
   return cudaGetLastError();
 }
 
