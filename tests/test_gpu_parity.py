@@ -739,6 +739,28 @@ def test_random_shapes_stress(seed):
     assert err <= TOL and lerr <= TOL, (kind, d, is_swa, err, lerr)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_many_rings_swa_decode(seed):
+    """Seeded random shapes with more rings than two, three or four per SM (the regimes of the compact single-token
+    ring kernel and its form with four blocks per SM): random window up to 128, page size, group size, head count,
+    ring heads and a mix of short and long contexts, every dead slot filled with +inf / NaN."""
+    rng = np.random.default_rng(7000 + seed)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    D = int(rng.choice([64, 128]))
+    P = int(rng.choice([16, 32, 64]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.choice([1, 2, 4]))
+    W = int(rng.choice([128, 128, 100, 64, 17]))
+    d = dims(G, D, P, Hkv, W=W)
+    per_sm = float(rng.choice([2.2, 3.3, 4.4]))
+    B = int(per_sm * sms / Hkv) + 1
+    ctx = [int(x) for x in np.where(rng.random(B) < 0.5, rng.integers(0, W + 3, B), rng.integers(W, 900, B))]
+    sc = build_scenario(d, ctx, [1] * B, seed=seed)
+    poison_dead_slots_nonfinite(sc)
+    err, lerr = run_decode(sc, True, bool(rng.integers(0, 2)))
+    assert err <= TOL and lerr <= TOL, (d, B, err, lerr)
+
+
 @pytest.mark.parametrize("sm_scale", [1.0, 3.0])
 def test_peaked_softmax_exercises_lazy_rescale(sm_scale):
     """Large score scale: row maxima keep growing from tile to tile by more than the 2^8 slack of the lazy
