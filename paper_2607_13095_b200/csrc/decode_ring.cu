@@ -543,6 +543,11 @@ decode_ring_compact_kernel(const __grid_constant__ RingMaps maps, const DecodePa
 // takes one m16n8k16 per 10 cycles); a ring is 144 such pairs.  Fragment loads are issued a granule ahead of the MMAs
 // that use them.
 // Stale rows (slots outside the window, granules not loaded) are masked in the scores and zeroed in the V fragments.
+// Second form (VE = 4, head_dim 128, between three and four rings per SM): only four V granules have a place of their
+// own, the others land in the K area once every compute warp has its scores, on a barrier of their own that every warp
+// waits on once per ring; 52 KB of tiles and 128 registers per thread, so four blocks fit an SM and no block walks a
+// second ring.  The next ring's loads then wait for the whole ring, which is why this form is not used beyond four rings
+// per SM.
 __device__ __forceinline__ void mma_inorder(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
