@@ -9,7 +9,7 @@ from oracle import hswa_oracle as orc
 from paper_2607_13095_b200 import binding as hb
 from paper_2607_13095_b200 import workloads as wl
 from helpers import build_scenario, oracle_config
-from gpu_utils import dev_batch, dev_i32, make_handle, to_dev_bf16, to_host_bits
+from gpu_utils import dev_batch, dev_i32, make_handle, to_dev_bf16, to_host_bits, workspace_for
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
@@ -209,3 +209,47 @@ def test_swa_prefill_is_repeatable_under_load():
     got = first.float().cpu().numpy()[tok, head]
     err = np.abs(got - ref)
     assert (err <= np.maximum(TOL, np.abs(ref) * 2.0 ** -8)).all(), float(err.max())
+
+
+@pytest.mark.parametrize("rings_per_sm", [3.3, 4.4], ids=["four_blocks_per_sm", "three_blocks_two_rounds"])
+def test_swa_decode_chain_is_repeatable(rings_per_sm):
+    """Chains of fused SWA decode calls on many rings, as a decode step issues them (six layers through one handle and
+    XX
+    output equals that of the first repetition bit for bit, no wait runs out, and the result agrees with the oracle.
+    The compact single-token ring kernel hands tiles between a loader warp and three compute warps over five barriers
+    (one of them only in its form with four blocks per SM); a wrong hand-off shows now and then, not every time."""
+    d = wl.BIG
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    B = int(rings_per_sm * sms / d.num_kv_heads) + 1
+    rng = np.random.default_rng(55)
+    ctx = [int(x) for x in rng.integers(100, 3000, B)]
+    sc = build_scenario(d, ctx, [1] * B, seed=55)
+    t = sc.tables
+    h = make_handle(d, out_dtype=torch.bfloat16)
+    b = dev_batch(t, decode=True)
+    layers = [hb.Layer(to_dev_bf16(sc.swa_pool), True) for _ in range(6)]
+    full = hb.Layer(to_dev_bf16(sc.full_pool), False)
+    q, k_new, v_new = to_dev_bf16(sc.q), to_dev_bf16(sc.k_new), to_dev_bf16(sc.v_new)
+    ws = workspace_for(h, t)
+    outs = [torch.zeros((B, d.num_q_heads, d.head_dim), dtype=torch.bfloat16, device="cuda") for _ in range(7)]
+    first = None
+    for rep in range(150):
+        if rep % 8 == 0:
+            hb.hswa_decode_attn(h, full, b, q, k_new, v_new, outs[6], None, ws)
+        for i, layer in enumerate(layers):
+            hb.hswa_decode_attn(h, layer, b, q, k_new, v_new, outs[i], None, ws)
+        torch.cuda.synchronize()
+        if first is None:
+            first = [o.clone() for o in outs[:6]]
+        else:
+            for i in range(6):
+                assert torch.equal(outs[i].view(torch.int16), first[i].view(torch.int16)), (rep, i)
+        for o in outs[:6]:
+            o.zero_()
+    async_err = hb.hswa_get_async_error(h)
+    assert async_err[0] == hb.HSWA_OK, async_err
+    ref, _ = orc.attention(sc.cfg, sc.layer(True), sc.batch(), sc.q, sc.k_new, sc.v_new)
+    for i in range(6):
+        assert torch.equal(first[i].view(torch.int16), first[0].view(torch.int16)), i
+    got = first[0].float().cpu().numpy().astype(np.float64)
+    assert np.abs(got - ref).max() <= 1e-2 + np.abs(ref).max() * 2.0 ** -8
