@@ -214,7 +214,7 @@ def test_swa_prefill_is_repeatable_under_load():
 @pytest.mark.parametrize("rings_per_sm", [3.3, 4.4], ids=["four_blocks_per_sm", "three_blocks_two_rounds"])
 def test_swa_decode_chain_is_repeatable(rings_per_sm):
     """Chains of fused SWA decode calls on many rings, as a decode step issues them (six layers through one handle and
-    XX
+    stream, each starting early behind the one before, a Full layer now and then), repeated 150 times: every layer's
     output equals that of the first repetition bit for bit, no wait runs out, and the result agrees with the oracle.
     The compact single-token ring kernel hands tiles between a loader warp and three compute warps over five barriers
     (one of them only in its form with four blocks per SM); a wrong hand-off shows now and then, not every time."""
